@@ -1,0 +1,260 @@
+"""Plain fp64 CPU oracle for attention with KV-cache eviction during prefilling
+and decoding (Batch-Max, Sec. 3: Algorithm 1 + the average-attention rule).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+benchmark's CPU-baseline leg.  It is slow on purpose, takes the algorithm's
+steps in the paper's order, and shares nothing with the CUDA path.
+
+The method is a heuristic whose result depends on the whole history of
+evictions, so the oracle *is* the algorithm, one step after the other, for one
+independent (layer, sample, kv-head) cache ("for each attention head and
+sample", Sec. 3.2).  All arithmetic is float64.
+
+Readings of points the paper leaves open (each is a convention of this build):
+  * "attention weights" are the post-softmax probabilities of causal scaled
+    dot-product attention with scale 1/sqrt(d) (Sec. 3.2 uses weights/scores
+    interchangeably).
+  * grouped-query attention (not mentioned in the paper): one cache and one
+    sum_weights vector per KV head; the weights of the g query heads of the
+    group are added, and ave_weights is divided by g so it stays in [0, 1].
+  * the denominator of ave_weights is the exact number of attention rows that
+    were accumulated for the pair, curr_id + 1 - kv_ids with curr_id the last
+    position processed (the justification given in Sec. 3.2, second paragraph).
+    Algorithm 1's literal decode-time curr_id (one larger) is available through
+    the ``curr_id`` argument of :meth:`UnitCache.evict`.
+  * ties in ave_weights: the pair with the lower position id is kept.
+  * survivors keep their sum_weights (the vector is "variable-sized": entries
+    leave with their pairs and nothing is reset).
+
+Parity unpinned (conventions, not derivable from the paper): the GQA sum, the
+tie direction and the denominator reading above.  Everything else is pinned by
+tests/test_oracle_pins.py.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+
+class UnitCache:
+    """KV cache of one (layer, sample, kv-head) with the eviction state of
+    Sec. 3.2: ``kv_ids`` (position ids, ascending), ``sum_weights`` and the
+    key/value rows themselves."""
+
+    def __init__(self, d: int, g: int = 1, scale: float | None = None):
+        self.d = int(d)
+        self.g = int(g)
+        self.scale = (1.0 / math.sqrt(d)) if scale is None else float(scale)
+        self.kv_ids = np.zeros(0, dtype=np.int64)
+        self.k = np.zeros((0, d), dtype=np.float64)
+        self.v = np.zeros((0, d), dtype=np.float64)
+        self.sum_weights = np.zeros(0, dtype=np.float64)
+        self.last_pos = -1            # curr_id: last position id processed
+        self.evicted_mass = 0.0       # sum_weights that left with evicted pairs
+        self.rows_processed = 0       # number of attention rows accumulated (queries x g)
+        self.last_eviction = None     # snapshot of the most recent eviction
+
+    def __len__(self) -> int:
+        return int(self.kv_ids.shape[0])
+
+    # ------------------------------------------------------------------ Sec. 3.2, update equation
+    def process_block(self, q, k, v, pos0: int, evict_to: int = -1, return_weights: bool = False):
+        """Forward pass with a block of ``I`` inputs at positions pos0..pos0+I-1.
+
+        q: (I, g, d)   k, v: (I, d).  Returns the attention output (I, g, d).
+        Every query attends to all cached pairs and to the block's pairs at
+        positions <= its own; sum_weights += sum_i attn_weights[i] (Sec. 3.2);
+        new pairs start from a zero sum_weights entry.  If ``evict_to >= 0``
+        and the cache is larger afterwards, it is cut back to ``evict_to``.
+        """
+        q = np.asarray(q, dtype=np.float64)
+        k = np.asarray(k, dtype=np.float64)
+        v = np.asarray(v, dtype=np.float64)
+        I = q.shape[0]
+        assert q.shape == (I, self.g, self.d) and k.shape == (I, self.d) and v.shape == (I, self.d)
+        if pos0 != self.last_pos + 1:
+            raise ValueError(f"pos0={pos0} does not follow last position {self.last_pos}")
+        n_old = len(self)
+        self.kv_ids = np.concatenate([self.kv_ids, pos0 + np.arange(I, dtype=np.int64)])
+        self.k = np.concatenate([self.k, k], axis=0)
+        self.v = np.concatenate([self.v, v], axis=0)
+        self.sum_weights = np.concatenate([self.sum_weights, np.zeros(I)])
+
+        out = np.zeros((I, self.g, self.d))
+        weights = np.zeros((I, self.g, n_old + I)) if return_weights else None
+        for i in range(I):
+            # visible pairs: every cached one, and the block's own up to position pos0 + i.
+            # kv_ids is ascending, so these are exactly the first m entries.
+            m = n_old + i + 1
+            assert self.kv_ids[m - 1] == pos0 + i
+            for h in range(self.g):
+                logits = self.scale * (self.k[:m] @ q[i, h])
+                w = np.exp(logits - logits.max())
+                w = w / w.sum()                      # attn_weights[i] for this head
+                out[i, h] = w @ self.v[:m]
+                self.sum_weights[:m] += w            # sum_weights += attn_weights[i]
+                if return_weights:
+                    weights[i, h, :m] = w
+        self.last_pos = pos0 + I - 1
+        self.rows_processed += I * self.g
+        if evict_to >= 0 and len(self) > evict_to:
+            self.evict(evict_to)
+        return (out, weights) if return_weights else out
+
+    def decode_step(self, q, k, v, evict_to: int = -1):
+        """One generated token: a block with I = 1 (Sec. 3.2: "during decoding I = 1").
+        q: (g, d), k, v: (d,).  Returns (g, d)."""
+        q = np.asarray(q, dtype=np.float64)[None]
+        k = np.asarray(k, dtype=np.float64)[None]
+        v = np.asarray(v, dtype=np.float64)[None]
+        return self.process_block(q, k, v, self.last_pos + 1, evict_to)[0]
+
+    # ------------------------------------------------------------------ Sec. 3.2, eviction rule
+    def ave_weights(self, curr_id: int | None = None):
+        """ave_weights = sum_weights / (curr_id + 1 - kv_ids), element-wise; divided by the
+        group size so a GQA group's summed weights stay in [0, 1]."""
+        curr_id = self.last_pos if curr_id is None else curr_id
+        count = curr_id + 1 - self.kv_ids
+        return self.sum_weights / (self.g * count)
+
+    def evict(self, target: int, curr_id: int | None = None, kept_ids=None):
+        """Remove the pairs with the smallest ave_weights until ``target`` remain.
+
+        Ranking: ave_weights descending, ties -> lower position id first; the first ``target``
+        survive and stay in ascending position order (stable compaction).  ``kept_ids`` overrides
+        the selection (used by lock-step parity to follow a choice made inside the tolerance
+        band); the snapshot in ``last_eviction`` always holds the oracle's own choice.
+        """
+        n = len(self)
+        target = int(target)
+        if target >= n:
+            return None
+        ave = self.ave_weights(curr_id)
+        order = np.lexsort((self.kv_ids, -ave))          # primary: -ave, secondary: id
+        own_keep = np.sort(order[:target])
+        cut = float(ave[order[target - 1]]) if target > 0 else math.inf
+        snap = {
+            "cand_ids": self.kv_ids.copy(),
+            "cand_ave": ave.copy(),
+            "cand_sum_weights": self.sum_weights.copy(),
+            "kept_ids": self.kv_ids[own_keep].copy(),
+            "cut": cut,
+            "target": target,
+        }
+        if kept_ids is None:
+            keep = own_keep
+        else:
+            kept_ids = np.asarray(kept_ids, dtype=np.int64)
+            assert kept_ids.shape[0] == target and np.all(np.diff(kept_ids) > 0)
+            keep = np.searchsorted(self.kv_ids, kept_ids)
+            assert np.array_equal(self.kv_ids[keep], kept_ids), "kept ids must be candidates"
+        gone = np.ones(n, dtype=bool)
+        gone[keep] = False
+        self.evicted_mass += float(self.sum_weights[gone].sum())
+        self.kv_ids = self.kv_ids[keep]
+        self.k = self.k[keep]
+        self.v = self.v[keep]
+        self.sum_weights = self.sum_weights[keep]
+        self.last_eviction = snap
+        return snap
+
+
+# ---------------------------------------------------------------------- plain definition
+def dense_causal_attention(q, k, v, scale: float | None = None):
+    """Full-KV-cache attention (the no-eviction limit, "FKV" in Sec. 4), written out from the
+    definition: out[i, h] = softmax_j<=i(scale * <q[i, h], k[j]>) . v.   q: (s, g, d), k, v: (s, d)."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    s, g, d = q.shape
+    scale = 1.0 / math.sqrt(d) if scale is None else scale
+    out = np.zeros((s, g, d))
+    for i in range(s):
+        for h in range(g):
+            logits = np.array([scale * float(np.dot(q[i, h], k[j])) for j in range(i + 1)])
+            w = np.exp(logits - logits.max())
+            w /= w.sum()
+            for j in range(i + 1):
+                out[i, h] += w[j] * v[j]
+    return out
+
+
+# ---------------------------------------------------------------------- schedules
+def _trace_entry(unit: UnitCache):
+    return unit.kv_ids.copy()
+
+
+def run_north_star(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec: int = 1,
+                   g: int | None = None, scale: float | None = None):
+    """Blocks of ``block`` prompt tokens (ragged tail allowed), the cache cut back to ``kv_max``
+    after every block; then ``steps`` decode steps, cut back to ``kv_max`` whenever the cache
+    has grown to ``kv_max + p_dec``.   q: (s+steps, g, d); k, v: (s+steps, d).
+    Returns (outputs (s+steps, g, d), trace of kv_ids after every call, unit)."""
+    q = np.asarray(q, dtype=np.float64)
+    g = q.shape[1] if g is None else g
+    unit = UnitCache(q.shape[2], g, scale)
+    outs, trace = [], []
+    pos = 0
+    while pos < s:
+        I = min(block, s - pos)
+        outs.append(unit.process_block(q[pos:pos + I], k[pos:pos + I], v[pos:pos + I], pos, kv_max))
+        trace.append(_trace_entry(unit))
+        pos += I
+    for t in range(steps):
+        full = len(unit) + 1 >= kv_max + p_dec
+        outs.append(unit.decode_step(q[s + t], k[s + t], v[s + t], kv_max if full else -1)[None])
+        trace.append(_trace_entry(unit))
+    return np.concatenate(outs, axis=0), trace, unit
+
+
+def run_algorithm1(q, k, v, s: int, kv_bar: int, p: int, max_gen: int, scale: float | None = None,
+                   literal_decode_curr_id: bool = False):
+    """Algorithm 1 as printed: first block of min(s, kv_bar) tokens; while tokens remain, remove p
+    pairs and process the next <= p tokens; then for t = 1..max_gen-1: if the cache holds kv_bar
+    pairs remove p, and process the token at position s + t - 1.
+    ``literal_decode_curr_id``: use the printed decode-time curr_id = s + t - 1 in the rule's
+    denominator (one more than the rows accumulated) instead of this build's reading."""
+    q = np.asarray(q, dtype=np.float64)
+    unit = UnitCache(q.shape[2], q.shape[1], scale)
+    outs, trace, sizes = [], [], []
+    t1 = min(s, kv_bar)
+    outs.append(unit.process_block(q[0:t1], k[0:t1], v[0:t1], 0))
+    trace.append(_trace_entry(unit))
+    while t1 < s:
+        unit.evict(len(unit) - p)
+        sizes.append(len(unit))
+        t0 = t1
+        t1 = min(s, t0 + p)
+        outs.append(unit.process_block(q[t0:t1], k[t0:t1], v[t0:t1], t0))
+        trace.append(_trace_entry(unit))
+    for t in range(1, max_gen):
+        if len(unit) == kv_bar:
+            unit.evict(len(unit) - p, curr_id=(s + t - 1) if literal_decode_curr_id else None)
+            sizes.append(len(unit))
+        pos = s + t - 1
+        outs.append(unit.decode_step(q[pos], k[pos], v[pos])[None])
+        trace.append(_trace_entry(unit))
+    return np.concatenate(outs, axis=0), trace, unit, sizes
+
+
+def run_decode_only(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec: int = 1,
+                    scale: float | None = None):
+    """Decoding-only compression (Sec. 1): the whole prompt is cached during prefilling (processed
+    here in blocks of ``block`` with no eviction), the cache is compressed to ``kv_max`` once after
+    the prompt, then decoding proceeds as in :func:`run_north_star`."""
+    q = np.asarray(q, dtype=np.float64)
+    unit = UnitCache(q.shape[2], q.shape[1], scale)
+    outs, trace = [], []
+    pos = 0
+    while pos < s:
+        I = min(block, s - pos)
+        outs.append(unit.process_block(q[pos:pos + I], k[pos:pos + I], v[pos:pos + I], pos))
+        pos += I
+    unit.evict(kv_max)
+    trace.append(_trace_entry(unit))
+    for t in range(steps):
+        full = len(unit) + 1 >= kv_max + p_dec
+        outs.append(unit.decode_step(q[s + t], k[s + t], v[s + t], kv_max if full else -1)[None])
+        trace.append(_trace_entry(unit))
+    return np.concatenate(outs, axis=0), trace, unit
