@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the Batch-Max evicting-attention hot path (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl ours|reference]
+
+A step is one pass of the whole path over one batch of the named workload: cache creation, every
+block-wise prefill call (attention, score reduction, top-k eviction with compaction) and every decode
+step (attention, score update, eviction).  `value` counts the tokens the batch pushed through the path
+(prompt + generated) per second with all inputs resident in HBM; `e2e` is the same pass through the
+host-fed entry points with pinned host buffers (copies inside the timed region).
+With N > 1 every rank runs an independent replica on its own GPU (the path has no exchange step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "P&D evicting-attention tokens/s at max batch; % of TC (prefill) / HBM (decode) peak"
+UNIT = "tokens/s"
+# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
+# capture, see profiles/); None until a capture of the current kernel exists.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"attn_fwd": None}
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------
+def workload_tokens(wl) -> int:
+    return wl.b * (wl.s + wl.steps) * wl.L
+
+
+def prefill_pairs(wl) -> int:
+    """Visible (query, key) pairs of one sample's q-head over the whole prompt schedule."""
+    n, pos, pairs = 0, 0, 0
+    while pos < wl.s:
+        I = min(wl.B, wl.s - pos)
+        pairs += I * n + I * (I + 1) // 2
+        n = min(n + I, wl.K)
+        pos += I
+    return pairs
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+                for nm, val in zip(names, r[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(nm)
+            except Exception:
+                continue
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+def run_reference(args, wl):
+    """The CPU oracle as it stands, timed on the host cores on a bounded sample of the workload."""
+    import numpy as np
+    import torch
+    from oracle import UnitCache
+    from paper_2412_05693_b200.workloads import Inputs, schedule
+    inp = Inputs(wl, "cpu")
+    calls = schedule(wl)
+    cores = torch.get_num_threads()
+
+    def one_unit(smp, kh, max_calls=None):
+        u = UnitCache(wl.d, wl.g)
+        t = 0.0
+        for kind, pos0, I, ev in calls[:max_calls]:
+            q, k, v = inp.block(0, pos0, I, smp, 1)
+            qq = q[0, :, kh * wl.g:(kh + 1) * wl.g].double().numpy()
+            kk, vv = k[0, :, kh].double().numpy(), v[0, :, kh].double().numpy()
+            t0 = time.perf_counter()
+            u.process_block(qq, kk, vv, pos0, ev)
+            t += time.perf_counter() - t0
+        return t
+
+    # size the sample: time one unit, then as many units as fit the budget per step
+    t_unit = one_unit(0, 0)
+    per_step_budget = max(args.cpu_seconds / max(1, args.steps + args.warmup), t_unit)
+    units_per_step = max(1, min(wl.b * wl.Hkv, int(per_step_budget / t_unit)))
+    unit_list = [(i % wl.b, (i // wl.b) % wl.Hkv) for i in range(units_per_step)]
+    times = []
+    for it in range(args.warmup + args.steps):
+        t = sum(one_unit(s, h) for s, h in unit_list)
+        if it >= args.warmup:
+            times.append(t)
+    t_mean = sum(times) / len(times)
+    tokens_per_unit = (wl.s + wl.steps) / wl.Hkv          # a sample's tokens are shared by its Hkv caches
+    value = units_per_step * tokens_per_unit / t_mean
+    sample = (f"{units_per_step} of {wl.b * wl.Hkv} (sample, kv-head) caches of layer 0, whole schedule each; "
+              f"tokens/s extrapolated linearly over caches (independent, equal cost)")
+    return value, t_mean * 1e3, cores, sample
+
+
+def cfg_dict(wl, extra=None):
+    d = {"workload": wl.name, "b": wl.b, "Hq": wl.Hq, "Hkv": wl.Hkv, "d": wl.d, "s": wl.s, "block": wl.B,
+         "kv_max": wl.K, "decode_steps": wl.steps, "layers": wl.L, "p_dec": wl.p_dec,
+         "l2": "flushed between timed steps (256 MiB write); per-step inputs exceed L2"}
+    if extra:
+        d.update(extra)
+    return d
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2412_05693_b200.workloads import WORKLOADS
+    wl = WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        value, ms, cores, sample = run_reference(args, wl)
+        line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "config": cfg_dict(wl),
+                "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+                "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+
+    import torch
+    import torch.distributed as dist
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    from paper_2412_05693_b200.build import build
+    if rank == 0 or world == 1:
+        build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    import paper_2412_05693_b200 as bm
+    from paper_2412_05693_b200.workloads import Inputs, schedule
+    from tests.lockstep import make_config
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    calls = schedule(wl)
+    cfg = make_config(wl, device=local_rank)
+    stream = torch.cuda.current_stream()
+
+    # ---- inputs resident in HBM (layer 0's stream is reused for every layer: layers are independent)
+    inp = Inputs(wl, dev)
+    dev_in = []
+    for kind, pos0, I, ev in calls:
+        q, k, v = inp.block(0, pos0, I)
+        if kind == "decode":
+            q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
+        dev_in.append((q, k, v))
+    out_blk = torch.empty(wl.b, wl.B, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
+    out_dec = torch.empty(wl.b, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
+    arena = torch.empty(bm.arena_bytes(cfg), dtype=torch.uint8, device=dev)
+    flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
+
+    def one_step(host_bufs=None):
+        cache = bm.BatchMaxCache(cfg, arena=arena)
+        for layer in range(wl.L):
+            for ci, (kind, pos0, I, ev) in enumerate(calls):
+                if host_bufs is None:
+                    q, k, v = dev_in[ci]
+                    if kind == "prefill":
+                        cache.prefill_block(q, k, v, pos0, out=out_blk[:, :I], evict_to=ev, layer=layer)
+                    else:
+                        cache.decode_step(q, k, v, out=out_dec, evict_to=ev, layer=layer)
+                else:
+                    q, k, v, o = host_bufs[ci]
+                    if kind == "prefill":
+                        cache.prefill_block_host(q, k, v, pos0, o, evict_to=ev, layer=layer)
+                    else:
+                        cache.decode_step_host(q, k, v, o, evict_to=ev, layer=layer)
+        return cache
+
+    def timed(n_warm, n_steps, host_bufs=None):
+        for _ in range(n_warm):
+            one_step(host_bufs).close()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ms = []
+        for _ in range(n_steps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            c = one_step(host_bufs)
+            e1.record(stream)
+            e1.synchronize()
+            c.close()
+            ms.append(e0.elapsed_time(e1))
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        total = torch.tensor([sum(ms)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(total, op=dist.ReduceOp.MAX)
+        return float(total.item()) / n_steps
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = bm.kernel_launch_count()
+    ms_step = timed(args.warmup, args.steps)
+    launches = (bm.kernel_launch_count() - launches0) // (args.warmup + args.steps) * args.steps
+    clocks = sampler.stop() if rank == 0 else None
+    tokens = workload_tokens(wl)
+    value = world * tokens / (ms_step * 1e-3)
+
+    # ---- dominant kernel: the prefill-block attention forward, timed per launch with CUDA events
+    prof = bm.binding.profile_pass(lambda: one_step().close()) if hasattr(bm.binding, "profile_pass") else None
+    pk, pk_src = peaks()
+    roofline = None
+    extra = {}
+    if prof is not None:
+        attn_ms, attn_n = prof["attn_fwd"]
+        flops_per_step = 4.0 * wl.d * prefill_pairs(wl) * wl.b * wl.Hq * wl.L
+        achieved = flops_per_step / (attn_ms * 1e-3) / 1e12 if attn_ms > 0 else 0.0
+        peak = pk["bf16_tflops_sustained"] if wl.dtype == "bf16" else pk["bf16_tflops_sustained"] / 2
+        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get("attn_fwd")
+        roofline = {"bound": "tensor", "kernel": "prefill-block attention forward", "achieved": achieved,
+                    "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic,
+                    "peak_source": f"{pk_src} (sustained bf16 matmul)", "launches_per_step": attn_n,
+                    "avg_launch_ms": attn_ms / max(attn_n, 1)}
+        extra["kernel_ms_per_step"] = {k: v[0] for k, v in prof.items()}
+        extra["kernel_launches_per_step"] = {k: v[1] for k, v in prof.items()}
+        dec_ms, dec_n = prof.get("decode", (0.0, 0))
+        if dec_ms > 0:
+            n1 = min(wl.K, wl.s) + 1
+            e = wl.elem_bytes
+            per_unit = n1 * 2 * wl.d * e + 16 * n1 + 2 * wl.d * e + 2 * wl.g * wl.d * e
+            dec_bytes = per_unit * wl.b * wl.Hkv * dec_n
+            gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
+            extra["decode_roofline"] = {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                                        "frac": gbs / pk["hbm_gbs"], "peak_source": pk_src,
+                                        "note": "algorithmic bytes without the compaction term"}
+
+    # ---- end to end through the host-fed entry points (pinned host inputs, outputs read back)
+    e2e = None
+    if not args.no_e2e:
+        host_bufs, h2d, d2h = [], 0, 0
+        for (q, k, v) in dev_in:
+            hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+            ho = torch.empty_like(hq).pin_memory()
+            host_bufs.append((hq, hk, hv, ho))
+            h2d += sum(t.numel() * t.element_size() for t in (hq, hk, hv))
+            d2h += ho.numel() * ho.element_size()
+        ms_e2e = timed(1, max(1, min(args.steps, 3)), host_bufs)
+        e2e = {"value": world * tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d * wl.L,
+               "d2h_bytes_per_step": d2h * wl.L, "ms_per_step": ms_e2e}
+        del host_bufs
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        a2 = argparse.Namespace(**vars(args))
+        a2.steps, a2.warmup = 1, 0
+        v, ms, cores, sample = run_reference(a2, wl)
+        cpu_baseline = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+
+    if rank == 0:
+        ppairs = prefill_pairs(wl) * wl.b * wl.Hq * wl.L
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+                "config": cfg_dict(wl, {"parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                                        "prefill_path": "tcgen05" if bm.last_prefill_path() == 1 else "simt-fp32"}),
+                "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
+                "clocks": clocks, "prefill_useful_tflop_per_step": 4.0 * wl.d * ppairs / 1e12}
+        line.update(extra)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

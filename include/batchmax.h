@@ -1,0 +1,187 @@
+/*
+ * batchmax.h -- C ABI of libbatchmax: attention with KV-cache eviction during
+ * prefilling and decoding (Batch-Max, arXiv 2412.05693) on one NVIDIA B200.
+ *
+ * Notation (Sec. 3 of the paper unless noted):
+ *   b        batch size (samples processed in parallel)
+ *   Hq, Hkv  query heads / KV heads, g = Hq / Hkv (g = 1 is plain multi-head)
+ *   d        head dimension
+ *   K        kv_max: size every (sample, kv-head) cache is cut back to by an
+ *            eviction.  Algorithm 1's limit \overline{|kv|} is K + p, its
+ *            eviction amount p is the growth allowed above K.
+ *   I        number of inputs (queries) in one forward pass; I = 1 in decoding
+ *   n        current number of KV pairs in a cache; n <= cap = K + growth
+ *   kv_ids, sum_weights, curr_id   as in Sec. 3.2
+ *
+ * General rules
+ *   - Every pointer argument is labelled HOST or DEVICE.  DEVICE pointers must
+ *     belong to cfg.device, be 16-byte aligned, and are only borrowed for the
+ *     stream-ordered duration of the call.  The library never allocates or
+ *     frees device memory: the cache lives in a caller-owned arena, per-call
+ *     scratch in a caller-owned workspace.
+ *   - Calls validate on the host, enqueue kernels on `cuda_stream`
+ *     (a cudaStream_t passed as void*, NULL = the legacy default stream) and
+ *     return without synchronising, except where stated.
+ *   - Every function returns a bm_status_t; nothing throws, aborts or traps.
+ *     On a non-BM_OK return nothing was enqueued and the cache is unchanged.
+ *   - A handle is not thread-safe; distinct handles are independent.
+ *   - All (sample, kv-head) caches of one (layer, sample) hold the same n, and
+ *     n after a call is a function of n before, I and evict_to only, so the
+ *     library mirrors n and curr_id on the host and never reads them back.
+ */
+#ifndef BATCHMAX_H_
+#define BATCHMAX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct bm_cache bm_cache_t; /* opaque, owned by the library */
+
+typedef enum {
+  BM_OK = 0,
+  BM_ERR_INVALID = 1,  /* null / negative / misaligned argument, unsupported shape        */
+  BM_ERR_OOM = 2,      /* arena, workspace or budget too small                            */
+  BM_ERR_CAPACITY = 3, /* the call would make n exceed cap, or too many candidates        */
+  BM_ERR_STATE = 4,    /* pos0 does not follow curr_id, or the sample range has unequal n */
+  BM_ERR_CUDA = 5,     /* a CUDA runtime or driver call failed                            */
+  BM_ERR_TIMEOUT = 6   /* a bounded device-side wait expired (see bm_cache_status)        */
+} bm_status_t;
+
+typedef enum { BM_F32 = 0, BM_BF16 = 1 } bm_dtype_t;
+
+/* Problem statement: Algorithm 1's inputs (\overline{|kv|}, p) generalised as (K, growth), plus the
+ * attention shape.  All sizes in elements. */
+typedef struct {
+  int32_t batch;            /* b                                                              */
+  int32_t n_layers;         /* L independent attention layers sharing the handle              */
+  int32_t n_q_heads;        /* Hq                                                             */
+  int32_t n_kv_heads;       /* Hkv, must divide Hq; g = Hq / Hkv <= 8                         */
+  int32_t head_dim;         /* d: 64 or 128                                                   */
+  int32_t kv_max;           /* K >= 1                                                         */
+  int32_t block_max;        /* largest I any bm_prefill_block call will pass, >= 1            */
+  int32_t growth;           /* G >= 1: rows above K a cache may hold between evictions        */
+  int32_t dtype;            /* bm_dtype_t of q/k/v/out and of the cached rows                 */
+  float softmax_scale;      /* 0 selects 1/sqrt(d)                                            */
+  int32_t device;           /* CUDA device ordinal                                            */
+  int32_t max_call_samples; /* largest nsamples of any call (sizes the workspace); 0 -> batch */
+} bm_config_t;
+
+/* ---- cache layout, allocator and memory model (Sec. 1: batch size under a fixed memory budget) ----
+ * Per sample the arena holds, for every layer and kv-head, cap = K + growth rows of:
+ * key (d elements), value (d elements), sum_weights (fp32) and kv_ids (int32):
+ *     bytes_per_sample = L * Hkv * cap * (2 * d * elem_size + 8).
+ * The arena adds a fixed 1024-byte header (status word, alignment of the four slabs). */
+bm_status_t bm_cache_bytes_per_sample(const bm_config_t* cfg /*HOST*/, size_t* bytes /*HOST out*/);
+/* Arena size for cfg->batch samples. */
+bm_status_t bm_arena_bytes(const bm_config_t* cfg /*HOST*/, size_t* bytes /*HOST out*/);
+/* Largest batch whose arena fits in hbm_budget_bytes (cfg->batch is ignored); 0 if none fits. */
+bm_status_t bm_max_batch(const bm_config_t* cfg /*HOST*/, size_t hbm_budget_bytes, int32_t* b /*HOST out*/);
+/* Per-call scratch (log-sum-exp of every query row and the new pairs' column sums) for calls of up
+ * to max_call_samples samples and block_max inputs. */
+bm_status_t bm_workspace_bytes(const bm_config_t* cfg /*HOST*/, size_t* bytes /*HOST out*/);
+
+/* Carve `arena` (DEVICE, 256-byte aligned, >= bm_arena_bytes) into the slabs
+ * K,V: [L][b][Hkv][cap][d], sum_weights: fp32 [L][b][Hkv][cap], kv_ids: int32 [L][b][Hkv][cap],
+ * zero it on `cuda_stream`, and return a handle with every cache empty (n = 0, curr_id = -1).
+ * `workspace` (DEVICE, 256-byte aligned, >= bm_workspace_bytes) is used by every later call; calls on
+ * the same handle must therefore be stream-ordered with respect to each other.
+ * Both buffers stay owned by the caller and must outlive the handle.
+ * Errors: BM_ERR_INVALID (bad config / null / misaligned), BM_ERR_OOM (a buffer is too small). */
+bm_status_t bm_cache_create(const bm_config_t* cfg /*HOST*/, void* arena /*DEVICE*/, size_t arena_bytes,
+                            void* workspace /*DEVICE*/, size_t workspace_bytes, void* cuda_stream,
+                            bm_cache_t** out /*HOST out*/);
+bm_status_t bm_cache_destroy(bm_cache_t* cache); /* frees the host handle only */
+
+/* ---- the forward pass with a block of I inputs (Sec. 3.2; Algorithm 1 "process tokens [t0, t1-1]") ----
+ * For samples sample0 .. sample0+nsamples-1 of `layer`: the I queries at positions pos0 .. pos0+I-1
+ * attend to all n cached pairs and to the block's own pairs at positions <= their own (causal);
+ *   out = softmax(scale * q k^T) v,      sum_weights += sum_i attn_weights[i]
+ * (summed over the g query heads of each KV head; new pairs start from 0), the block's pairs join the
+ * cache with kv_ids = their positions, curr_id becomes pos0+I-1.  Then, if evict_to >= 0 and
+ * n + I > evict_to, the caches are cut back to evict_to pairs exactly as bm_evict does.
+ *   q   DEVICE [nsamples][I][Hq][d]     k, v  DEVICE [nsamples][I][Hkv][d]    (contiguous, cfg.dtype)
+ *   out DEVICE [nsamples][I][Hq][d]     (cfg.dtype)
+ * The block's K/V are read from the caller's buffers (they are not staged in the cache first), so the
+ * call needs min(n + I, evict_to if evicting) <= cap, not n + I <= cap.
+ * Errors: BM_ERR_INVALID (range, I < 1, I > block_max, null, misaligned), BM_ERR_STATE (pos0 !=
+ * curr_id + 1, or the samples of the range hold different n), BM_ERR_CAPACITY. */
+bm_status_t bm_prefill_block(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples,
+                             const void* q, const void* k, const void* v, int32_t I, int32_t pos0,
+                             void* out, int32_t evict_to, void* cuda_stream);
+
+/* ---- one decoding step (Algorithm 1 "generate token"; Sec. 3.2 "during decoding I = 1") ----
+ * Same as bm_prefill_block with I = 1 and pos0 = curr_id + 1, in one bandwidth-bound pass.
+ *   q, out DEVICE [nsamples][Hq][d]     k, v DEVICE [nsamples][Hkv][d]
+ * Needs n + 1 <= cap (the new pair is appended before an optional eviction). */
+bm_status_t bm_decode_step(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples,
+                           const void* q, const void* k, const void* v, void* out, int32_t evict_to,
+                           void* cuda_stream);
+
+/* ---- eviction (Algorithm 1 "remove p KV pairs"; Sec. 3.2 average-attention rule) ----
+ * For every (sample, kv-head) of the range independently:
+ *   ave_weights = sum_weights / (g * (curr_id + 1 - kv_ids));
+ * keep the `target` pairs that rank first under (ave_weights descending, kv_ids ascending), move them
+ * to the front of the cache in ascending kv_ids order together with their sum_weights and kv_ids,
+ * n becomes target.  No-op when n <= target.  Errors: BM_ERR_INVALID (target < 0, range), BM_ERR_STATE. */
+bm_status_t bm_evict(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples, int32_t target,
+                     void* cuda_stream);
+
+/* ---- the same two passes fed from HOST memory (end-to-end use without device-side producers) ----
+ * q/k/v/out are HOST pointers (pinned memory makes the copies asynchronous); `staging` is a DEVICE
+ * buffer of at least bm_staging_bytes(cfg, nsamples, I) bytes.  The call copies q, k, v to the device,
+ * runs the pass, copies out back to `out` -- all on cuda_stream -- and does not synchronise. */
+bm_status_t bm_staging_bytes(const bm_config_t* cfg /*HOST*/, int32_t nsamples, int32_t I, size_t* bytes);
+bm_status_t bm_prefill_block_host(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples,
+                                  const void* q /*HOST*/, const void* k /*HOST*/, const void* v /*HOST*/,
+                                  int32_t I, int32_t pos0, void* out /*HOST*/, int32_t evict_to,
+                                  void* staging /*DEVICE*/, size_t staging_bytes, void* cuda_stream);
+bm_status_t bm_decode_step_host(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples,
+                                const void* q /*HOST*/, const void* k /*HOST*/, const void* v /*HOST*/,
+                                void* out /*HOST*/, int32_t evict_to, void* staging /*DEVICE*/,
+                                size_t staging_bytes, void* cuda_stream);
+
+/* ---- state access ---- */
+/* Host mirror of n and curr_id (-1 when empty) of one (layer, sample); no synchronisation. */
+bm_status_t bm_cache_len(const bm_cache_t* cache, int32_t layer, int32_t sample, int32_t* n /*HOST out*/,
+                         int32_t* curr_id /*HOST out, may be NULL*/);
+/* Copy one (layer, sample, kv-head) cache to HOST arrays: kv_ids[n], sum_weights[n] and, when not
+ * NULL, k_rows / v_rows [n][d] in cfg.dtype.  Synchronises cuda_stream before returning. */
+bm_status_t bm_cache_export(bm_cache_t* cache, int32_t layer, int32_t sample, int32_t kv_head,
+                            int32_t* kv_ids /*HOST out*/, float* sum_weights /*HOST out*/,
+                            void* k_rows /*HOST out*/, void* v_rows /*HOST out*/, int32_t* n /*HOST out*/,
+                            void* cuda_stream);
+/* Inverse of bm_cache_export for checkpoint / resume: overwrite the first n rows of one
+ * (layer, sample, kv-head) cache; n must equal the mirrored n of that sample (set it first with
+ * bm_cache_set_len).  Synchronises cuda_stream before returning. */
+bm_status_t bm_cache_import(bm_cache_t* cache, int32_t layer, int32_t sample, int32_t kv_head,
+                            const int32_t* kv_ids /*HOST*/, const float* sum_weights /*HOST*/,
+                            const void* k_rows /*HOST*/, const void* v_rows /*HOST*/, int32_t n,
+                            void* cuda_stream);
+/* Set the mirrored n (0 <= n <= cap) and curr_id of one (layer, sample) when restoring a checkpoint. */
+bm_status_t bm_cache_set_len(bm_cache_t* cache, int32_t layer, int32_t sample, int32_t n, int32_t curr_id);
+/* Synchronise cuda_stream and read the device status word: BM_OK, or BM_ERR_TIMEOUT if a kernel gave
+ * up a bounded wait (its results are then undefined; the context stays usable). */
+bm_status_t bm_cache_status(bm_cache_t* cache, int32_t* device_status /*HOST out*/, void* cuda_stream);
+
+/* ---- per-kernel timing (measurement aid; the paper has no counterpart) ----
+ * While enabled, every kernel launch of this library is bracketed by two CUDA events on its stream.
+ * bm_profile_read waits for the recorded launches of one kernel class, returns their summed duration in
+ * milliseconds and their count, and forgets them.  Not thread-safe; leave disabled in production. */
+enum { BM_KERNEL_ATTN_FWD = 0, BM_KERNEL_SCORE = 1, BM_KERNEL_EVICT = 2, BM_KERNEL_DECODE = 3 };
+bm_status_t bm_profile_enable(int32_t on);
+bm_status_t bm_profile_read(int32_t kernel_class, float* total_ms /*HOST out*/, int32_t* launches /*HOST out*/);
+
+/* Number of kernels this library has launched in the calling process (monotone counter). */
+uint64_t bm_kernel_launch_count(void);
+/* Which attention implementation the last bm_prefill_block used: 0 = fp32 SIMT, 1 = tcgen05 bf16. */
+int32_t bm_last_prefill_path(void);
+const char* bm_status_string(bm_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BATCHMAX_H_ */

@@ -1,0 +1,522 @@
+// Host side of the C ABI: memory model and allocator (arena carving), argument validation, the host
+// mirror of n / curr_id, and the stream-ordered launch sequence of every entry point.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <utility>
+#include <vector>
+
+#include "../../include/batchmax.h"
+#include "common.cuh"
+
+namespace bm {
+unsigned long long g_launch_count = 0;
+int g_last_prefill_path = 0;
+
+namespace {
+bool g_profile_on = false;
+std::vector<cudaEvent_t> g_event_pool;
+std::vector<std::pair<cudaEvent_t, cudaEvent_t>> g_pairs[kNumKernelClasses];
+cudaEvent_t g_open_start = nullptr;
+cudaEvent_t take_event() {
+  if (!g_event_pool.empty()) { cudaEvent_t e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+}  // namespace
+
+void profile_begin(int, cudaStream_t st) {
+  if (!g_profile_on) return;
+  g_open_start = take_event();
+  if (g_open_start) cudaEventRecord(g_open_start, st);
+}
+void profile_end(int cls, cudaStream_t st) {
+  if (!g_profile_on || g_open_start == nullptr) return;
+  cudaEvent_t stop = take_event();
+  if (stop) cudaEventRecord(stop, st);
+  g_pairs[cls].push_back({g_open_start, stop});
+  g_open_start = nullptr;
+}
+}  // namespace bm
+
+using namespace bm;
+
+namespace {
+
+constexpr size_t kHeaderBytes = 1024;   // status word + room to align each of the four slabs to 256 B
+constexpr int kMaxCandidates = 12288;   // candidates of one eviction must fit one CTA's shared memory
+constexpr size_t kMaxSmem = 227 * 1024;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline size_t elem_size(int dtype) { return dtype == BM_BF16 ? 2 : 4; }
+
+bool config_ok(const bm_config_t* c, bool need_batch) {
+  if (c == nullptr) return false;
+  if (need_batch && c->batch < 1) return false;
+  if (c->n_layers < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1) return false;
+  if (c->n_q_heads % c->n_kv_heads != 0) return false;
+  const int g = c->n_q_heads / c->n_kv_heads;
+  if (!(g == 1 || g == 2 || g == 4 || g == 8)) return false;
+  if (!(c->head_dim == 64 || c->head_dim == 128)) return false;
+  if (c->kv_max < 1 || c->block_max < 1 || c->growth < 1) return false;
+  if (!(c->dtype == BM_F32 || c->dtype == BM_BF16)) return false;
+  if (!(c->softmax_scale >= 0.f) || std::isinf(c->softmax_scale)) return false;
+  if (c->device < 0 || c->max_call_samples < 0) return false;
+  if ((long long)c->kv_max + c->growth > (1 << 24)) return false;
+  return true;
+}
+
+size_t per_sample_bytes(const bm_config_t* c) {
+  const size_t cap = (size_t)c->kv_max + c->growth;
+  return (size_t)c->n_layers * c->n_kv_heads * cap * (2 * (size_t)c->head_dim * elem_size(c->dtype) + 8);
+}
+
+int call_samples(const bm_config_t* c) { return c->max_call_samples > 0 ? c->max_call_samples : c->batch; }
+
+size_t ws_lse_bytes(const bm_config_t* c) {
+  return align_up(sizeof(float) * (size_t)call_samples(c) * c->n_q_heads * c->block_max, 256);
+}
+size_t ws_newsum_bytes(const bm_config_t* c) {
+  return align_up(sizeof(float) * (size_t)call_samples(c) * c->n_kv_heads * c->block_max, 256);
+}
+
+}  // namespace
+
+struct bm_cache {
+  bm_config_t cfg;
+  int cap, g;
+  size_t esz;
+  float scale;
+  char* k_slab;
+  char* v_slab;
+  float* sum_weights;
+  int32_t* kv_ids;
+  int32_t* status;
+  float* ws_lse;
+  float* ws_new_sum;
+  std::vector<int32_t> n, curr_id;  // [L * b] host mirror
+};
+
+namespace {
+
+bm_status_t set_device(const bm_cache* c) {
+  return cudaSetDevice(c->cfg.device) == cudaSuccess ? BM_OK : BM_ERR_CUDA;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Range checks shared by the per-call entry points; returns the common n of the range in *n.
+bm_status_t check_range(const bm_cache* c, int layer, int sample0, int nsamples, int* n, int* curr) {
+  if (c == nullptr) return BM_ERR_INVALID;
+  if (layer < 0 || layer >= c->cfg.n_layers) return BM_ERR_INVALID;
+  if (sample0 < 0 || nsamples < 1 || (long long)sample0 + nsamples > c->cfg.batch) return BM_ERR_INVALID;
+  if (nsamples > call_samples(&c->cfg)) return BM_ERR_INVALID;
+  const size_t o = (size_t)layer * c->cfg.batch + sample0;
+  for (int s = 1; s < nsamples; ++s)
+    if (c->n[o + s] != c->n[o] || c->curr_id[o + s] != c->curr_id[o]) return BM_ERR_STATE;
+  *n = c->n[o];
+  *curr = c->curr_id[o];
+  return BM_OK;
+}
+
+CacheView make_view(const bm_cache* c, int layer, int sample0, int nsamples, int n_old) {
+  CacheView v;
+  const size_t unit0 = ((size_t)layer * c->cfg.batch + sample0) * c->cfg.n_kv_heads;
+  const size_t row0 = unit0 * c->cap;
+  v.k_slab = c->k_slab + row0 * c->cfg.head_dim * c->esz;
+  v.v_slab = c->v_slab + row0 * c->cfg.head_dim * c->esz;
+  v.sum_weights = c->sum_weights + row0;
+  v.kv_ids = c->kv_ids + row0;
+  v.cap = c->cap;
+  v.n_old = n_old;
+  v.Hq = c->cfg.n_q_heads;
+  v.Hkv = c->cfg.n_kv_heads;
+  v.g = c->g;
+  v.nsamples = nsamples;
+  v.status = c->status;
+  return v;
+}
+
+void set_mirror(bm_cache* c, int layer, int sample0, int nsamples, int n, int curr) {
+  const size_t o = (size_t)layer * c->cfg.batch + sample0;
+  for (int s = 0; s < nsamples; ++s) { c->n[o + s] = n; c->curr_id[o + s] = curr; }
+}
+
+}  // namespace
+
+extern "C" {
+
+bm_status_t bm_cache_bytes_per_sample(const bm_config_t* cfg, size_t* bytes) {
+  if (!config_ok(cfg, false) || bytes == nullptr) return BM_ERR_INVALID;
+  *bytes = per_sample_bytes(cfg);
+  return BM_OK;
+}
+
+bm_status_t bm_arena_bytes(const bm_config_t* cfg, size_t* bytes) {
+  if (!config_ok(cfg, true) || bytes == nullptr) return BM_ERR_INVALID;
+  *bytes = kHeaderBytes + per_sample_bytes(cfg) * (size_t)cfg->batch;
+  return BM_OK;
+}
+
+bm_status_t bm_max_batch(const bm_config_t* cfg, size_t hbm_budget_bytes, int32_t* b) {
+  if (!config_ok(cfg, false) || b == nullptr) return BM_ERR_INVALID;
+  if (hbm_budget_bytes <= kHeaderBytes) { *b = 0; return BM_OK; }
+  const size_t q = (hbm_budget_bytes - kHeaderBytes) / per_sample_bytes(cfg);
+  *b = (int32_t)(q > 0x7fffffff ? 0x7fffffff : q);
+  return BM_OK;
+}
+
+bm_status_t bm_workspace_bytes(const bm_config_t* cfg, size_t* bytes) {
+  if (!config_ok(cfg, true) || bytes == nullptr) return BM_ERR_INVALID;
+  *bytes = ws_lse_bytes(cfg) + ws_newsum_bytes(cfg);
+  return BM_OK;
+}
+
+bm_status_t bm_cache_create(const bm_config_t* cfg, void* arena, size_t arena_bytes, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream, bm_cache_t** out) {
+  if (!config_ok(cfg, true) || arena == nullptr || workspace == nullptr || out == nullptr) return BM_ERR_INVALID;
+  if ((reinterpret_cast<uintptr_t>(arena) & 255u) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return BM_ERR_INVALID;
+  size_t need_arena = 0, need_ws = 0;
+  bm_arena_bytes(cfg, &need_arena);
+  bm_workspace_bytes(cfg, &need_ws);
+  if (arena_bytes < need_arena || workspace_bytes < need_ws) return BM_ERR_OOM;
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return BM_ERR_CUDA;
+
+  bm_cache* c = new (std::nothrow) bm_cache();
+  if (c == nullptr) return BM_ERR_OOM;
+  c->cfg = *cfg;
+  c->cap = cfg->kv_max + cfg->growth;
+  c->g = cfg->n_q_heads / cfg->n_kv_heads;
+  c->esz = elem_size(cfg->dtype);
+  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+  const size_t rows = (size_t)cfg->n_layers * cfg->batch * cfg->n_kv_heads * c->cap;
+  const size_t slab = rows * cfg->head_dim * c->esz;  // multiple of 128 bytes
+  char* p = static_cast<char*>(arena);
+  c->status = reinterpret_cast<int32_t*>(p);
+  // header = 256 B status block + up to 3 * 256 B of slab alignment padding
+  size_t off = 256;
+  c->k_slab = p + off;                                   off = align_up(off + slab, 256);
+  c->v_slab = p + off;                                   off = align_up(off + slab, 256);
+  c->sum_weights = reinterpret_cast<float*>(p + off);    off = align_up(off + rows * 4, 256);
+  c->kv_ids = reinterpret_cast<int32_t*>(p + off);       off += rows * 4;
+  if (off > need_arena) { delete c; return BM_ERR_OOM; }
+  c->ws_lse = static_cast<float*>(workspace);
+  c->ws_new_sum = reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_lse_bytes(cfg));
+  c->n.assign((size_t)cfg->n_layers * cfg->batch, 0);
+  c->curr_id.assign((size_t)cfg->n_layers * cfg->batch, -1);
+  // Unwritten rows are read as zero-weight padding by the tiled kernels, so they must hold finite values.
+  if (cudaMemsetAsync(arena, 0, need_arena, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+    delete c;
+    return BM_ERR_CUDA;
+  }
+  *out = c;
+  return BM_OK;
+}
+
+bm_status_t bm_cache_destroy(bm_cache_t* cache) {
+  if (cache == nullptr) return BM_ERR_INVALID;
+  delete cache;
+  return BM_OK;
+}
+
+static bm_status_t run_evict(bm_cache* c, const CacheView& view, const EvictArgs& e, cudaStream_t st) {
+  if (evict_smem_bytes(view.n_old + e.I, e.target) > kMaxSmem) return BM_ERR_CAPACITY;
+  return launch_evict(c->cfg.dtype, c->cfg.head_dim, view, e, st) == cudaSuccess ? BM_OK : BM_ERR_CUDA;
+}
+
+bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, const void* q,
+                             const void* k, const void* v, int32_t I, int32_t pos0, void* out,
+                             int32_t evict_to, void* cuda_stream) {
+  int n_old = 0, curr = 0;
+  bm_status_t s = check_range(c, layer, sample0, nsamples, &n_old, &curr);
+  if (s != BM_OK) return s;
+  if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) return BM_ERR_INVALID;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BM_ERR_INVALID;
+  if (I < 1 || I > c->cfg.block_max) return BM_ERR_INVALID;
+  if (pos0 != curr + 1) return BM_ERR_STATE;
+  const int n_c = n_old + I;
+  const int target = (evict_to >= 0 && n_c > evict_to) ? evict_to : n_c;
+  if (target > c->cap) return BM_ERR_CAPACITY;
+  if (n_c > kMaxCandidates || evict_smem_bytes(n_c, target) > kMaxSmem) return BM_ERR_CAPACITY;
+  if ((s = set_device(c)) != BM_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+  CacheView view = make_view(c, layer, sample0, nsamples, n_old);
+  BlockArgs a;
+  a.q = q; a.k = k; a.v = v; a.out = out;
+  a.lse = c->ws_lse; a.new_sum = c->ws_new_sum;
+  a.I = I; a.pos0 = pos0; a.scale = c->scale;
+
+  int used_tc = 0;
+  if (c->cfg.dtype == BM_BF16 && tc_path_available()) {
+    if (launch_attn_tc(c->cfg.head_dim, view, a, st, &used_tc) != cudaSuccess) return BM_ERR_CUDA;
+  }
+  if (!used_tc && launch_attn_simt(c->cfg.dtype, c->cfg.head_dim, view, a, st) != cudaSuccess) return BM_ERR_CUDA;
+  g_last_prefill_path = used_tc;
+  int used_tc_score = 0;
+  if (c->cfg.dtype == BM_BF16 && tc_path_available()) {
+    if (launch_score_tc(c->cfg.head_dim, view, a, st, &used_tc_score) != cudaSuccess) return BM_ERR_CUDA;
+  }
+  if (!used_tc_score && launch_score_simt(c->cfg.dtype, c->cfg.head_dim, view, a, st) != cudaSuccess)
+    return BM_ERR_CUDA;
+
+  int n_new = 0;
+  if (target > 0) {
+    EvictArgs e;
+    e.blk_k = k; e.blk_v = v; e.new_sum = c->ws_new_sum;
+    e.I = I; e.pos0 = pos0; e.curr_id = pos0 + I - 1; e.target = target;
+    if ((s = run_evict(c, view, e, st)) != BM_OK) return s;
+    n_new = target;
+  }
+  set_mirror(c, layer, sample0, nsamples, n_new, pos0 + I - 1);
+  return BM_OK;
+}
+
+bm_status_t bm_decode_step(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, const void* q,
+                           const void* k, const void* v, void* out, int32_t evict_to, void* cuda_stream) {
+  int n_old = 0, curr = 0;
+  bm_status_t s = check_range(c, layer, sample0, nsamples, &n_old, &curr);
+  if (s != BM_OK) return s;
+  if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) return BM_ERR_INVALID;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BM_ERR_INVALID;
+  const int n1 = n_old + 1;
+  if (n1 > c->cap) return BM_ERR_CAPACITY;
+  const int target = (evict_to >= 0 && n1 > evict_to) ? evict_to : -1;
+  if (n1 > kMaxCandidates || decode_smem_bytes(c->cfg.head_dim, c->g, n1, target) > kMaxSmem) return BM_ERR_CAPACITY;
+  if ((s = set_device(c)) != BM_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CacheView view = make_view(c, layer, sample0, nsamples, n_old);
+  const int pos = curr + 1;
+  int n_new = n1;
+  if (target == 0) {
+    // nothing survives: run the attention and the update, then empty the caches on the host mirror
+    if (launch_decode(c->cfg.dtype, c->cfg.head_dim, view, q, k, v, out, pos, c->scale, -1, st) != cudaSuccess)
+      return BM_ERR_CUDA;
+    n_new = 0;
+  } else {
+    if (launch_decode(c->cfg.dtype, c->cfg.head_dim, view, q, k, v, out, pos, c->scale, target, st) != cudaSuccess)
+      return BM_ERR_CUDA;
+    if (target > 0) n_new = target;
+  }
+  set_mirror(c, layer, sample0, nsamples, n_new, pos);
+  return BM_OK;
+}
+
+bm_status_t bm_evict(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, int32_t target,
+                     void* cuda_stream) {
+  int n_old = 0, curr = 0;
+  bm_status_t s = check_range(c, layer, sample0, nsamples, &n_old, &curr);
+  if (s != BM_OK) return s;
+  if (target < 0) return BM_ERR_INVALID;
+  if (n_old <= target) return BM_OK;
+  if (target == 0) { set_mirror(c, layer, sample0, nsamples, 0, curr); return BM_OK; }
+  if (n_old > kMaxCandidates) return BM_ERR_CAPACITY;
+  if ((s = set_device(c)) != BM_OK) return s;
+  CacheView view = make_view(c, layer, sample0, nsamples, n_old);
+  EvictArgs e;
+  e.blk_k = nullptr; e.blk_v = nullptr; e.new_sum = nullptr;
+  e.I = 0; e.pos0 = 0; e.curr_id = curr; e.target = target;
+  if ((s = run_evict(c, view, e, static_cast<cudaStream_t>(cuda_stream))) != BM_OK) return s;
+  set_mirror(c, layer, sample0, nsamples, target, curr);
+  return BM_OK;
+}
+
+// ---- host-fed variants ---------------------------------------------------------------------------
+static void staging_layout(const bm_config_t* cfg, int nsamples, int I, size_t* oq, size_t* ok, size_t* ov,
+                           size_t* oo, size_t* total, size_t* qbytes, size_t* kbytes) {
+  const size_t e = elem_size(cfg->dtype);
+  *qbytes = (size_t)nsamples * I * cfg->n_q_heads * cfg->head_dim * e;
+  *kbytes = (size_t)nsamples * I * cfg->n_kv_heads * cfg->head_dim * e;
+  size_t off = 0;
+  *oq = off; off = align_up(off + *qbytes, 256);
+  *ok = off; off = align_up(off + *kbytes, 256);
+  *ov = off; off = align_up(off + *kbytes, 256);
+  *oo = off; off = align_up(off + *qbytes, 256);
+  *total = off;
+}
+
+bm_status_t bm_staging_bytes(const bm_config_t* cfg, int32_t nsamples, int32_t I, size_t* bytes) {
+  if (!config_ok(cfg, false) || nsamples < 1 || I < 1 || bytes == nullptr) return BM_ERR_INVALID;
+  size_t oq, ok, ov, oo, qb, kb;
+  staging_layout(cfg, nsamples, I, &oq, &ok, &ov, &oo, bytes, &qb, &kb);
+  return BM_OK;
+}
+
+static bm_status_t host_pass(bm_cache_t* c, int layer, int sample0, int nsamples, const void* q, const void* k,
+                             const void* v, int I, int pos0, void* out, int evict_to, void* staging,
+                             size_t staging_bytes, void* cuda_stream, bool decode) {
+  int n_old = 0, curr = 0;
+  bm_status_t s = check_range(c, layer, sample0, nsamples, &n_old, &curr);
+  if (s != BM_OK) return s;
+  if (q == nullptr || k == nullptr || v == nullptr || out == nullptr || staging == nullptr) return BM_ERR_INVALID;
+  if (reinterpret_cast<uintptr_t>(staging) & 255u) return BM_ERR_INVALID;
+  if (I < 1 || I > c->cfg.block_max) return BM_ERR_INVALID;
+  size_t oq, ok, ov, oo, total, qb, kb;
+  staging_layout(&c->cfg, nsamples, I, &oq, &ok, &ov, &oo, &total, &qb, &kb);
+  if (staging_bytes < total) return BM_ERR_OOM;
+  // validate the pass itself before any copy is enqueued
+  if (decode) {
+    if (n_old + 1 > c->cap) return BM_ERR_CAPACITY;
+  } else {
+    if (pos0 != curr + 1) return BM_ERR_STATE;
+    const int n_c = n_old + I;
+    const int target = (evict_to >= 0 && n_c > evict_to) ? evict_to : n_c;
+    if (target > c->cap || n_c > kMaxCandidates || evict_smem_bytes(n_c, target) > kMaxSmem) return BM_ERR_CAPACITY;
+  }
+  if ((s = set_device(c)) != BM_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  char* sp = static_cast<char*>(staging);
+  if (cudaMemcpyAsync(sp + oq, q, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return BM_ERR_CUDA;
+  if (cudaMemcpyAsync(sp + ok, k, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return BM_ERR_CUDA;
+  if (cudaMemcpyAsync(sp + ov, v, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return BM_ERR_CUDA;
+  s = decode ? bm_decode_step(c, layer, sample0, nsamples, sp + oq, sp + ok, sp + ov, sp + oo, evict_to, cuda_stream)
+             : bm_prefill_block(c, layer, sample0, nsamples, sp + oq, sp + ok, sp + ov, I, pos0, sp + oo, evict_to,
+                                cuda_stream);
+  if (s != BM_OK) return s;
+  if (cudaMemcpyAsync(out, sp + oo, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return BM_ERR_CUDA;
+  return BM_OK;
+}
+
+bm_status_t bm_prefill_block_host(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, const void* q,
+                                  const void* k, const void* v, int32_t I, int32_t pos0, void* out,
+                                  int32_t evict_to, void* staging, size_t staging_bytes, void* cuda_stream) {
+  return host_pass(c, layer, sample0, nsamples, q, k, v, I, pos0, out, evict_to, staging, staging_bytes,
+                   cuda_stream, false);
+}
+
+bm_status_t bm_decode_step_host(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, const void* q,
+                                const void* k, const void* v, void* out, int32_t evict_to, void* staging,
+                                size_t staging_bytes, void* cuda_stream) {
+  return host_pass(c, layer, sample0, nsamples, q, k, v, 1, 0, out, evict_to, staging, staging_bytes, cuda_stream,
+                   true);
+}
+
+// ---- state access ----------------------------------------------------------------------------------
+bm_status_t bm_cache_len(const bm_cache_t* c, int32_t layer, int32_t sample, int32_t* n, int32_t* curr_id) {
+  if (c == nullptr || n == nullptr) return BM_ERR_INVALID;
+  if (layer < 0 || layer >= c->cfg.n_layers || sample < 0 || sample >= c->cfg.batch) return BM_ERR_INVALID;
+  const size_t o = (size_t)layer * c->cfg.batch + sample;
+  *n = c->n[o];
+  if (curr_id != nullptr) *curr_id = c->curr_id[o];
+  return BM_OK;
+}
+
+bm_status_t bm_cache_set_len(bm_cache_t* c, int32_t layer, int32_t sample, int32_t n, int32_t curr_id) {
+  if (c == nullptr) return BM_ERR_INVALID;
+  if (layer < 0 || layer >= c->cfg.n_layers || sample < 0 || sample >= c->cfg.batch) return BM_ERR_INVALID;
+  if (n < 0 || n > c->cap || curr_id < -1) return BM_ERR_INVALID;
+  const size_t o = (size_t)layer * c->cfg.batch + sample;
+  c->n[o] = n;
+  c->curr_id[o] = curr_id;
+  return BM_OK;
+}
+
+static bm_status_t unit_offsets(const bm_cache* c, int layer, int sample, int kv_head, size_t* row0) {
+  if (c == nullptr) return BM_ERR_INVALID;
+  if (layer < 0 || layer >= c->cfg.n_layers || sample < 0 || sample >= c->cfg.batch) return BM_ERR_INVALID;
+  if (kv_head < 0 || kv_head >= c->cfg.n_kv_heads) return BM_ERR_INVALID;
+  *row0 = (((size_t)layer * c->cfg.batch + sample) * c->cfg.n_kv_heads + kv_head) * c->cap;
+  return BM_OK;
+}
+
+bm_status_t bm_cache_export(bm_cache_t* c, int32_t layer, int32_t sample, int32_t kv_head, int32_t* kv_ids,
+                            float* sum_weights, void* k_rows, void* v_rows, int32_t* n, void* cuda_stream) {
+  size_t row0 = 0;
+  bm_status_t s = unit_offsets(c, layer, sample, kv_head, &row0);
+  if (s != BM_OK) return s;
+  if (n == nullptr) return BM_ERR_INVALID;
+  if ((s = set_device(c)) != BM_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int cnt = c->n[(size_t)layer * c->cfg.batch + sample];
+  *n = cnt;
+  const size_t rb = (size_t)c->cfg.head_dim * c->esz;
+  bool ok = true;
+  if (cnt > 0) {
+    if (kv_ids) ok &= cudaMemcpyAsync(kv_ids, c->kv_ids + row0, 4 * (size_t)cnt, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (sum_weights) ok &= cudaMemcpyAsync(sum_weights, c->sum_weights + row0, 4 * (size_t)cnt, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (k_rows) ok &= cudaMemcpyAsync(k_rows, c->k_slab + row0 * rb, rb * cnt, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (v_rows) ok &= cudaMemcpyAsync(v_rows, c->v_slab + row0 * rb, rb * cnt, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  }
+  ok &= cudaStreamSynchronize(st) == cudaSuccess;
+  return ok ? BM_OK : BM_ERR_CUDA;
+}
+
+bm_status_t bm_cache_import(bm_cache_t* c, int32_t layer, int32_t sample, int32_t kv_head, const int32_t* kv_ids,
+                            const float* sum_weights, const void* k_rows, const void* v_rows, int32_t n,
+                            void* cuda_stream) {
+  size_t row0 = 0;
+  bm_status_t s = unit_offsets(c, layer, sample, kv_head, &row0);
+  if (s != BM_OK) return s;
+  if (kv_ids == nullptr || sum_weights == nullptr || k_rows == nullptr || v_rows == nullptr) return BM_ERR_INVALID;
+  if (n != c->n[(size_t)layer * c->cfg.batch + sample]) return BM_ERR_STATE;
+  if ((s = set_device(c)) != BM_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t rb = (size_t)c->cfg.head_dim * c->esz;
+  bool ok = true;
+  if (n > 0) {
+    ok &= cudaMemcpyAsync(c->kv_ids + row0, kv_ids, 4 * (size_t)n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(c->sum_weights + row0, sum_weights, 4 * (size_t)n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(c->k_slab + row0 * rb, k_rows, rb * n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok &= cudaMemcpyAsync(c->v_slab + row0 * rb, v_rows, rb * n, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  }
+  ok &= cudaStreamSynchronize(st) == cudaSuccess;
+  return ok ? BM_OK : BM_ERR_CUDA;
+}
+
+bm_status_t bm_cache_status(bm_cache_t* c, int32_t* device_status, void* cuda_stream) {
+  if (c == nullptr || device_status == nullptr) return BM_ERR_INVALID;
+  bm_status_t s = set_device(c);
+  if (s != BM_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int32_t w = 0;
+  if (cudaMemcpyAsync(&w, c->status, sizeof(w), cudaMemcpyDeviceToHost, st) != cudaSuccess) return BM_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return BM_ERR_CUDA;
+  *device_status = w;
+  return BM_OK;
+}
+
+bm_status_t bm_profile_enable(int32_t on) {
+  g_profile_on = on != 0;
+  return BM_OK;
+}
+
+bm_status_t bm_profile_read(int32_t kernel_class, float* total_ms, int32_t* launches) {
+  if (kernel_class < 0 || kernel_class >= kNumKernelClasses || total_ms == nullptr || launches == nullptr)
+    return BM_ERR_INVALID;
+  float tot = 0.f;
+  int cnt = 0;
+  bool ok = true;
+  for (auto& pr : g_pairs[kernel_class]) {
+    float ms = 0.f;
+    if (pr.first && pr.second && cudaEventSynchronize(pr.second) == cudaSuccess &&
+        cudaEventElapsedTime(&ms, pr.first, pr.second) == cudaSuccess) { tot += ms; ++cnt; }
+    else ok = false;
+    if (pr.first) g_event_pool.push_back(pr.first);
+    if (pr.second) g_event_pool.push_back(pr.second);
+  }
+  g_pairs[kernel_class].clear();
+  *total_ms = tot;
+  *launches = cnt;
+  return ok ? BM_OK : BM_ERR_CUDA;
+}
+
+uint64_t bm_kernel_launch_count(void) { return (uint64_t)g_launch_count; }
+int32_t bm_last_prefill_path(void) { return g_last_prefill_path; }
+
+const char* bm_status_string(bm_status_t s) {
+  switch (s) {
+    case BM_OK: return "ok";
+    case BM_ERR_INVALID: return "invalid argument";
+    case BM_ERR_OOM: return "arena, workspace or budget too small";
+    case BM_ERR_CAPACITY: return "cache capacity or candidate limit exceeded";
+    case BM_ERR_STATE: return "call out of order for the cache state";
+    case BM_ERR_CUDA: return "CUDA call failed";
+    case BM_ERR_TIMEOUT: return "bounded device wait expired";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

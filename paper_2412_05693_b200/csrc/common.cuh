@@ -1,0 +1,97 @@
+// Shared declarations of the CUDA path: cache view, launcher prototypes, small device helpers.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace bm {
+
+// Device-side view of one layer's slabs for a contiguous range of samples (Sec. 3: one cache per
+// attention head and sample).  Unit u = local_sample * Hkv + kv_head; its rows start at u * cap.
+struct CacheView {
+  void* k_slab;        // [units][cap][d] elements of the cache dtype
+  void* v_slab;        // [units][cap][d]
+  float* sum_weights;  // [units][cap]
+  int32_t* kv_ids;     // [units][cap]
+  int32_t cap;
+  int32_t n_old;       // pairs cached before this call (equal for every unit of the range)
+  int32_t Hq, Hkv, g;
+  int32_t nsamples;
+  int32_t* status;     // device status word
+};
+
+// One forward pass over a block (I inputs) for the range.
+struct BlockArgs {
+  const void* q;    // [nsamples][I][Hq][d]
+  const void* k;    // [nsamples][I][Hkv][d]
+  const void* v;    // [nsamples][I][Hkv][d]
+  void* out;        // [nsamples][I][Hq][d]
+  float* lse;       // workspace: [units][I*g]  natural-log-sum-exp of every query row
+  float* new_sum;   // workspace: [units][I]    column sums of the block's own pairs
+  int32_t I;
+  int32_t pos0;
+  float scale;
+};
+
+struct EvictArgs {
+  const void* blk_k;     // block K/V when the new pairs still live in the caller's buffers, else null
+  const void* blk_v;
+  const float* new_sum;  // [units][I] when I > 0
+  int32_t I;             // candidates = n_old + I
+  int32_t pos0;
+  int32_t curr_id;       // last processed position
+  int32_t target;        // pairs to keep (<= n_old + I)
+};
+
+// Launchers (host).  All enqueue on `st` and return the CUDA error of the launch.
+cudaError_t launch_attn_simt(int dtype, int d, const CacheView& c, const BlockArgs& a, cudaStream_t st);
+cudaError_t launch_score_simt(int dtype, int d, const CacheView& c, const BlockArgs& a, cudaStream_t st);
+cudaError_t launch_evict(int dtype, int d, const CacheView& c, const EvictArgs& e, cudaStream_t st);
+cudaError_t launch_decode(int dtype, int d, const CacheView& c, const void* q, const void* k, const void* v,
+                          void* out, int32_t pos, float scale, int32_t target /* <0: none */, cudaStream_t st);
+size_t evict_smem_bytes(int n_cand, int target);
+size_t decode_smem_bytes(int d, int g, int n_rows, int target);
+bool tc_path_available();
+cudaError_t launch_attn_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used);
+cudaError_t launch_score_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used);
+
+extern unsigned long long g_launch_count;
+inline void count_launch(int n = 1) { g_launch_count += (unsigned long long)n; }
+
+// Optional per-launch timing: when enabled, a ProfileScope brackets a launch with two CUDA events.
+enum KernelClass { kAttnFwd = 0, kScore = 1, kEvict = 2, kDecode = 3, kNumKernelClasses = 4 };
+void profile_begin(int cls, cudaStream_t st);
+void profile_end(int cls, cudaStream_t st);
+struct ProfileScope {
+  int cls; cudaStream_t st;
+  ProfileScope(int c, cudaStream_t s) : cls(c), st(s) { profile_begin(cls, st); }
+  ~ProfileScope() { profile_end(cls, st); }
+};
+
+// ---- element helpers -------------------------------------------------------------------------
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static constexpr int kVec = 4;  // elements per 16-byte load
+  __device__ static inline void unpack(const uint4& r, float* f) {
+    f[0] = __uint_as_float(r.x); f[1] = __uint_as_float(r.y);
+    f[2] = __uint_as_float(r.z); f[3] = __uint_as_float(r.w);
+  }
+  __device__ static inline float to_out(float x) { return x; }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static constexpr int kVec = 8;
+  __device__ static inline void unpack(const uint4& r, float* f) {
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {  // bf16 -> fp32 is a 16-bit shift
+      f[2 * i] = __uint_as_float(w[i] << 16);
+      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  __device__ static inline __nv_bfloat16 to_out(float x) { return __float2bfloat16_rn(x); }
+};
+
+__device__ inline uint4 ld_global_16(const void* p) { return *reinterpret_cast<const uint4*>(p); }
+__device__ inline void st_global_16(void* p, const uint4& v) { *reinterpret_cast<uint4*>(p) = v; }
+
+}  // namespace bm

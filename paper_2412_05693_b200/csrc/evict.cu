@@ -1,0 +1,44 @@
+// Stand-alone eviction kernel: one CTA per (sample, kv-head) cache.  Used after a prefill block
+// (candidates = cached pairs + the block's pairs) and by bm_evict (candidates = cached pairs).
+#include "evict.cuh"
+
+namespace bm {
+namespace {
+
+constexpr int kEvictThreads = 512;
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kEvictThreads) evict_kernel(CacheView c, EvictArgs e) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int unit = blockIdx.x;
+  evict_body<T, D, kEvictThreads>(c, unit, unit / c.Hkv, unit % c.Hkv, e, smem_raw);
+}
+
+template <typename T, int D>
+cudaError_t launch_t(const CacheView& c, const EvictArgs& e, cudaStream_t st) {
+  const size_t smem = evict_smem_bytes(c.n_old + e.I, e.target);
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaError_t err = cudaFuncSetAttribute(evict_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    configured = smem;
+  }
+  ProfileScope prof(kEvict, st);
+  evict_kernel<T, D><<<c.nsamples * c.Hkv, kEvictThreads, smem, st>>>(c, e);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+size_t evict_smem_bytes(int n_cand, int target) { return evict_smem_layout(nullptr, n_cand, target, nullptr); }
+
+cudaError_t launch_evict(int dtype, int d, const CacheView& c, const EvictArgs& e, cudaStream_t st) {
+  if (dtype == 0 && d == 64) return launch_t<float, 64>(c, e, st);
+  if (dtype == 0 && d == 128) return launch_t<float, 128>(c, e, st);
+  if (dtype == 1 && d == 64) return launch_t<__nv_bfloat16, 64>(c, e, st);
+  if (dtype == 1 && d == 128) return launch_t<__nv_bfloat16, 128>(c, e, st);
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace bm

@@ -1,0 +1,203 @@
+// Average-attention eviction for one (sample, kv-head) cache, executed by one CTA (Sec. 3.2):
+//   ave_weights = sum_weights / (g * (curr_id + 1 - kv_ids)),
+// keep the `target` candidates ranking first under (ave_weights descending, kv_ids ascending),
+// then compact rows, sum_weights and kv_ids to the front of the cache in ascending kv_ids order.
+// Candidates are the n_old cached pairs followed by I new pairs that still live in the caller's
+// block buffers; both lists are ascending in kv_ids, so candidate index order is kv_ids order.
+#pragma once
+#include "common.cuh"
+
+namespace bm {
+
+struct EvictSmem {
+  float* score;    // [n_cand]
+  int32_t* id;     // [n_cand]
+  int32_t* src;    // [target]   candidate index that lands in row r
+  uint32_t* hist;  // [256]
+  int32_t* misc;   // [8]
+  int32_t* wsum;   // [64]
+};
+
+__host__ __device__ inline size_t evict_smem_layout(unsigned char* base, int n_cand, int target, EvictSmem* s) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) & ~size_t(15); return o; };
+  size_t o_score = take(sizeof(float) * n_cand), o_id = take(sizeof(int32_t) * n_cand);
+  size_t o_src = take(sizeof(int32_t) * (target > 0 ? target : 1)), o_hist = take(sizeof(uint32_t) * 256);
+  size_t o_misc = take(sizeof(int32_t) * 8), o_wsum = take(sizeof(int32_t) * 64);
+  if (s != nullptr) {
+    s->score = reinterpret_cast<float*>(base + o_score);
+    s->id = reinterpret_cast<int32_t*>(base + o_id);
+    s->src = reinterpret_cast<int32_t*>(base + o_src);
+    s->hist = reinterpret_cast<uint32_t*>(base + o_hist);
+    s->misc = reinterpret_cast<int32_t*>(base + o_misc);
+    s->wsum = reinterpret_cast<int32_t*>(base + o_wsum);
+  }
+  return off;
+}
+
+// Exclusive block scan of two counters packed per thread; returns this thread's exclusive prefixes.
+template <int NT>
+__device__ inline void block_exclusive_scan2(int a, int b, int32_t* wsum /*[64]*/, int& ea, int& eb) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int ia = a, ib = b;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int ta = __shfl_up_sync(0xffffffffu, ia, off), tb = __shfl_up_sync(0xffffffffu, ib, off);
+    if (lane >= off) { ia += ta; ib += tb; }
+  }
+  if (lane == 31) { wsum[warp] = ia; wsum[32 + warp] = ib; }
+  __syncthreads();
+  int ba = 0, bb = 0;
+  for (int w = 0; w < warp; ++w) { ba += wsum[w]; bb += wsum[32 + w]; }
+  ea = ba + ia - a;
+  eb = bb + ib - b;
+  __syncthreads();
+}
+
+template <typename T, int D, int NT>
+__device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh, const EvictArgs& e,
+                                  unsigned char* smem_raw) {
+  const int tid = threadIdx.x;
+  const int n_old = c.n_old, n_c = c.n_old + e.I, target = e.target;
+  const size_t base = (size_t)unit * c.cap;
+  EvictSmem s;
+  evict_smem_layout(smem_raw, n_c, target, &s);
+
+  for (int j = tid; j < n_c; j += NT) {
+    if (j < n_old) { s.score[j] = c.sum_weights[base + j]; s.id[j] = c.kv_ids[base + j]; }
+    else { s.score[j] = e.new_sum[(size_t)unit * e.I + (j - n_old)]; s.id[j] = e.pos0 + (j - n_old); }
+  }
+  __syncthreads();
+  const float gf = (float)c.g;
+  auto ave_bits = [&](int j) -> uint32_t {
+    const float cnt = (float)(e.curr_id + 1 - s.id[j]);
+    return __float_as_uint(s.score[j] / (gf * cnt));  // ave >= 0, so the bit pattern orders like the value
+  };
+
+  if (target >= n_c) {
+    for (int r = tid; r < n_c; r += NT) s.src[r] = r;
+    __syncthreads();
+  } else {
+    // ---- radix select: bit pattern `thr` of the target-th largest ave, and how many equal to it to keep
+    uint32_t prefix = 0, mask = 0;
+    int need = target;
+    for (int pass = 0; pass < 4; ++pass) {
+      const int shift = 24 - 8 * pass;
+      for (int t = tid; t < 256; t += NT) s.hist[t] = 0;
+      __syncthreads();
+      for (int j = tid; j < n_c; j += NT) {
+        const uint32_t b = ave_bits(j);
+        if ((b & mask) == prefix) atomicAdd(&s.hist[(b >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (tid < 32) {  // lane l owns digits 8l .. 8l+7; find the digit holding the need-th largest
+        int loc = 0;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) loc += (int)s.hist[tid * 8 + t];
+        int incl = loc;  // suffix sums over lanes above
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int t = __shfl_down_sync(0xffffffffu, incl, off);
+          if (tid + off < 32) incl += t;
+        }
+        const int above = incl - loc;
+        if (above < need && need <= above + loc) {
+          int cum = above, dg = 7;
+          for (; dg >= 0; --dg) {
+            const int h = (int)s.hist[tid * 8 + dg];
+            if (cum + h >= need) break;
+            cum += h;
+          }
+          s.misc[0] = tid * 8 + dg;
+          s.misc[1] = need - cum;
+        }
+      }
+      __syncthreads();
+      prefix |= ((uint32_t)s.misc[0]) << shift;
+      mask |= 255u << shift;
+      need = s.misc[1];
+      __syncthreads();
+    }
+    const uint32_t thr = prefix;
+    const int need_eq = need;
+    // ---- stable destinations: candidates above thr, plus the first need_eq equal to thr (lower id first)
+    const int chunk = (n_c + NT - 1) / NT;
+    const int jb = min(tid * chunk, n_c), je = min(jb + chunk, n_c);
+    int gt = 0, eq = 0;
+    for (int j = jb; j < je; ++j) {
+      const uint32_t b = ave_bits(j);
+      gt += (b > thr);
+      eq += (b == thr);
+    }
+    int gt_before, eq_before;
+    block_exclusive_scan2<NT>(gt, eq, s.wsum, gt_before, eq_before);
+    for (int j = jb; j < je; ++j) {
+      const uint32_t b = ave_bits(j);
+      if (b > thr) { s.src[gt_before + min(eq_before, need_eq)] = j; ++gt_before; }
+      else if (b == thr) {
+        if (eq_before < need_eq) s.src[gt_before + eq_before] = j;
+        ++eq_before;
+      }
+    }
+    __syncthreads();
+  }
+
+  // ---- first row that changes (rows before it keep their place and their contents)
+  if (tid == 0) s.misc[2] = target;
+  __syncthreads();
+  {
+    int first = target;
+    for (int r = tid; r < target; r += NT)
+      if (s.src[r] != r || s.src[r] >= n_old) { first = r; break; }
+    if (first < target) atomicMin(&s.misc[2], first);
+  }
+  __syncthreads();
+  const int first_moved = s.misc[2];
+
+  for (int r = first_moved + tid; r < target; r += NT) {
+    const int j = s.src[r];
+    c.sum_weights[base + r] = s.score[j];
+    c.kv_ids[base + r] = s.id[j];
+  }
+
+  // ---- rows: ascending chunks, every source row index >= its destination, loads of a chunk complete
+  // (barrier) before its stores; later chunks only read rows above everything written so far.
+  constexpr int PR = D * (int)sizeof(T) / 16;  // 16-byte pieces per row
+  constexpr int U = 4;                         // pieces per thread per tensor and chunk
+  constexpr int RC = NT * U / PR;              // rows per chunk
+  T* kslab = reinterpret_cast<T*>(c.k_slab) + base * D;
+  T* vslab = reinterpret_cast<T*>(c.v_slab) + base * D;
+  for (int r0 = first_moved; r0 < target; r0 += RC) {
+    uint4 kb[U], vb[U];
+    bool mv[U];
+#pragma unroll
+    for (int t = 0; t < U; ++t) {
+      const int pidx = t * NT + tid, r = r0 + pidx / PR, pc = pidx % PR;
+      mv[t] = false;
+      if (r < target) {
+        const int j = s.src[r];
+        if (j >= n_old) {
+          const size_t off = ((size_t)(smp * e.I + (j - n_old)) * c.Hkv + kh) * D;
+          kb[t] = ld_global_16(reinterpret_cast<const T*>(e.blk_k) + off + pc * (16 / sizeof(T)));
+          vb[t] = ld_global_16(reinterpret_cast<const T*>(e.blk_v) + off + pc * (16 / sizeof(T)));
+          mv[t] = true;
+        } else if (j != r) {
+          kb[t] = ld_global_16(kslab + (size_t)j * D + pc * (16 / sizeof(T)));
+          vb[t] = ld_global_16(vslab + (size_t)j * D + pc * (16 / sizeof(T)));
+          mv[t] = true;
+        }
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int t = 0; t < U; ++t) {
+      if (mv[t]) {
+        const int pidx = t * NT + tid, r = r0 + pidx / PR, pc = pidx % PR;
+        st_global_16(kslab + (size_t)r * D + pc * (16 / sizeof(T)), kb[t]);
+        st_global_16(vslab + (size_t)r * D + pc * (16 / sizeof(T)), vb[t]);
+      }
+    }
+  }
+}
+
+}  // namespace bm

@@ -1,0 +1,114 @@
+"""Lock-step parity driver: runs a workload's schedule through the C-ABI library on the GPU and through the
+fp64 oracle on the same input bits, call by call, for a chosen set of (sample, kv-head) caches.
+
+Free-running comparison is meaningless after the first near-tie (one flipped choice changes every later kept
+set), so after each call the GPU's kept ids are checked against the oracle's *own* ranking:
+  - every candidate whose ave_weights is above cut*(1+band) must be kept, none below cut*(1-band) may be,
+    the kept count equals the target and ids ascend;
+  - if the sets differ only inside the band, the oracle adopts the GPU's set (keeping its own fp64 sums)
+    and the adoption is counted.
+Outputs are compared on every call, sum_weights after every call, and cached K/V rows bit for bit.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import UnitCache
+from paper_2412_05693_b200 import BatchMaxCache, Config
+from paper_2412_05693_b200.workloads import Inputs, Workload, schedule
+
+BAND = 1e-4   # relative band around the cut inside which kept sets may differ
+OUT_TOL = {"bf16": 2e-2, "f32": 1e-4}
+
+
+def make_config(wl: Workload, device: int = 0, growth: int | None = None, batch: int | None = None,
+                max_call_samples: int = 0) -> Config:
+    return Config(batch=wl.b if batch is None else batch, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.d,
+                  kv_max=wl.K, block_max=wl.B, growth=max(1, wl.p_dec) if growth is None else growth,
+                  dtype=wl.dtype, n_layers=wl.L, device=device, max_call_samples=max_call_samples)
+
+
+def _np(t):
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def check_kept(unit: UnitCache, gpu_ids: np.ndarray, target: int, stats: dict, where: str):
+    """Band check of the GPU's kept set against the oracle's ranking; the oracle then evicts (adopting the
+    GPU's set when it differs inside the band)."""
+    ave = unit.ave_weights()
+    cand = unit.kv_ids
+    order = np.lexsort((cand, -ave))
+    cut = ave[order[target - 1]]
+    gpu = np.asarray(gpu_ids, dtype=np.int64)
+    assert gpu.shape[0] == target, f"{where}: kept {gpu.shape[0]} != target {target}"
+    assert np.all(np.diff(gpu) > 0), f"{where}: kept ids not ascending"
+    in_cand = np.isin(gpu, cand)
+    assert in_cand.all(), f"{where}: kept ids that were never candidates: {gpu[~in_cand][:8]}"
+    kept_mask = np.isin(cand, gpu)
+    must_keep = ave > cut * (1 + BAND)
+    must_drop = ave < cut * (1 - BAND)
+    assert not np.any(must_keep & ~kept_mask), f"{where}: dropped a pair clearly above the cut"
+    assert not np.any(must_drop & kept_mask), f"{where}: kept a pair clearly below the cut"
+    own = cand[np.sort(order[:target])]
+    if not np.array_equal(own, gpu):
+        stats["adoptions"] += 1
+    unit.evict(target, kept_ids=gpu)
+    stats["evictions"] += 1
+
+
+def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=None, check_rows_every: int = 8,
+                 growth: int | None = None, sum_rtol: float | None = None):
+    """Run `calls` (default: the workload's spec schedule) on the GPU for the whole batch and on the
+    oracle for `units` = [(sample, kv_head), ...].  Returns a dict of statistics; raises on any mismatch."""
+    dev = torch.device("cuda", device)
+    inp = Inputs(wl, dev)
+    cfg = make_config(wl, device, growth)
+    cache = BatchMaxCache(cfg)
+    g = wl.g
+    oracles = {u: UnitCache(wl.d, g) for u in units}
+    stats = {"adoptions": 0, "evictions": 0, "max_out_err": 0.0, "max_sum_rel": 0.0, "calls": 0, "tc_calls": 0}
+    tol = OUT_TOL[wl.dtype]
+    sum_rtol = sum_rtol if sum_rtol is not None else (2e-3 if wl.dtype == "bf16" else 2e-4)
+    calls = schedule(wl) if calls is None else calls
+    from paper_2412_05693_b200 import last_prefill_path
+    for ci, (kind, pos0, I, evict_to) in enumerate(calls):
+        if kind == "evict":
+            cache.evict(evict_to, layer=layer)
+            q = k = v = out = None
+        else:
+            q, k, v = inp.block(layer, pos0, I)
+            if kind == "prefill":
+                out = cache.prefill_block(q, k, v, pos0, evict_to=evict_to, layer=layer)
+                stats["tc_calls"] += last_prefill_path()
+            else:
+                out = cache.decode_step(q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous(),
+                                        evict_to=evict_to, layer=layer)[:, None]
+        torch.cuda.synchronize(dev)
+        assert cache.status() == 0
+        stats["calls"] += 1
+        for (smp, kh), unit in oracles.items():
+            where = f"call {ci} ({kind} pos0={pos0} I={I}) unit ({smp},{kh})"
+            if kind != "evict":
+                ref = unit.process_block(_np(q[smp, :, kh * g:(kh + 1) * g]), _np(k[smp, :, kh]), _np(v[smp, :, kh]),
+                                         pos0, -1)
+                err = float(np.abs(_np(out[smp, :, kh * g:(kh + 1) * g]) - ref).max())
+                stats["max_out_err"] = max(stats["max_out_err"], err)
+                assert err <= tol, f"{where}: output max-abs error {err:.3e} > {tol}"
+            want_rows = (ci % check_rows_every == 0) or ci == len(calls) - 1
+            ids, sw, kr, vr = cache.export(layer, smp, kh, rows=want_rows)
+            ids = ids.numpy().astype(np.int64)
+            if evict_to >= 0 and len(unit) > evict_to:
+                check_kept(unit, ids, evict_to, stats, where)
+            assert np.array_equal(ids, unit.kv_ids), f"{where}: kv_ids differ from the oracle's"
+            n_gpu, cur = cache.length(layer, smp)
+            assert n_gpu == len(unit) and cur == unit.last_pos, f"{where}: host mirror n/curr_id wrong"
+            sw = sw.numpy().astype(np.float64)
+            rel = float(np.max(np.abs(sw - unit.sum_weights) / np.maximum(np.abs(unit.sum_weights), 1e-3)))
+            stats["max_sum_rel"] = max(stats["max_sum_rel"], rel)
+            assert rel <= sum_rtol, f"{where}: sum_weights relative error {rel:.3e} > {sum_rtol}"
+            if want_rows:
+                assert np.array_equal(_np(kr), unit.k), f"{where}: cached K rows are not the oracle's rows"
+                assert np.array_equal(_np(vr), unit.v), f"{where}: cached V rows are not the oracle's rows"
+    cache.close()
+    return stats

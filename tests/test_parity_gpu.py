@@ -1,0 +1,249 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle in lock-step on the same
+seeded inputs.  Kept sets bit-exact outside a 1e-4 relative band around the cut, outputs within 2e-2 (bf16) /
+1e-4 (fp32) max-abs, cached rows bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2412_05693_b200 as bm
+from paper_2412_05693_b200.workloads import CFG5_SWEEP, WORKLOADS, Inputs, Workload, schedule
+from tests.lockstep import make_config, run_lockstep
+
+pytestmark = pytest.mark.gpu
+
+
+def all_units(wl, samples=None):
+    samples = range(wl.b) if samples is None else samples
+    return [(s, h) for s in samples for h in range(wl.Hkv)]
+
+
+def tiny(name, **kw):
+    base = dict(b=2, Hq=4, Hkv=2, d=64, dtype="f32", s=200, B=48, K=40, steps=6, seed=123, heavy_count=4)
+    base.update(kw)
+    return Workload(name, **base)
+
+
+# ------------------------------------------------------------------ configs of the benchmark table
+def test_cfg1_everything():
+    wl = WORKLOADS["cfg1"]
+    st = run_lockstep(wl, all_units(wl), check_rows_every=1)
+    assert st["evictions"] >= (6 + 16) * 8
+    assert st["max_out_err"] <= 1e-4
+
+
+def test_cfg2_full_size_sampled_units():
+    wl = WORKLOADS["cfg2"]
+    st = run_lockstep(wl, [(0, 0), (7, 3), (15, 7)], check_rows_every=16)
+    assert st["evictions"] > 0 and st["max_out_err"] <= 2e-2
+
+
+def test_cfg3_full_size_sampled_units():
+    wl = WORKLOADS["cfg3"].with_(steps=8)
+    run_lockstep(wl, [(3, 1), (12, 6)], check_rows_every=8)
+
+
+def test_cfg3_decode_only_compression_arm():
+    # whole prompt cached (cap = s + 1), one compression to K after the prompt, then decode (Sec. 1)
+    wl = WORKLOADS["cfg3"].with_(b=2, s=2048, steps=4)
+    calls = [("prefill", p, wl.B, -1) for p in range(0, wl.s, wl.B)] + [("evict", 0, 0, wl.K)]
+    calls += [("decode", wl.s + t, 1, wl.K) for t in range(wl.steps)]
+    run_lockstep(wl, [(0, 0), (1, 5)], calls=calls, growth=wl.s + 1 - wl.K)
+
+
+def test_cfg4_layers_are_independent():
+    wl = WORKLOADS["cfg4"].with_(b=2, L=3, s=2048, steps=3)
+    for layer in (0, 2):
+        run_lockstep(wl, [(1, 2)], layer=layer, check_rows_every=4)
+
+
+@pytest.mark.parametrize("B,K", [CFG5_SWEEP[1], CFG5_SWEEP[3], CFG5_SWEEP[5]])
+def test_cfg5_large_candidate_sets(B, K):
+    wl = WORKLOADS["cfg5"].with_(b=2, B=B, K=K, s=8192, steps=4)
+    run_lockstep(wl, [(1, 17)], check_rows_every=4)
+
+
+# ------------------------------------------------------------------ shapes, tails and degenerate cases
+@pytest.mark.parametrize("wl", [
+    tiny("ragged_f32"),                                               # I = 48, tail of 8, g = 2
+    tiny("gqa8_bf16", Hq=16, Hkv=2, dtype="bf16", d=128, B=50, K=70, s=333),
+    tiny("mha_bf16_d64", Hq=3 * 1, Hkv=3, dtype="bf16", d=64, B=64, K=64, s=256),
+    tiny("block_gt_cache", B=96, K=16, s=300),                        # B > K: no Algorithm-1 counterpart
+    tiny("short_prompt", s=30, B=16, K=64, steps=40),                 # s < K: eviction starts in decode
+    tiny("one_token_blocks", s=40, B=1, K=8, steps=3),
+    tiny("keep_one", s=64, B=16, K=1, steps=5),
+    tiny("f32_d128_g4", Hq=8, Hkv=2, d=128, B=40, K=100, s=260),
+    tiny("decode_growth", p_dec=8, s=96, B=32, K=32, steps=30),       # evict every 8th step
+], ids=lambda w: w.name)
+def test_small_shapes(wl):
+    st = run_lockstep(wl, all_units(wl), check_rows_every=1)
+    assert st["calls"] == len(schedule(wl))
+
+
+def test_algorithm1_cadence_on_gpu():
+    # Algorithm 1 as printed: limit kv_bar, remove p before each block / when full during decoding
+    kv_bar, p, s, gen = 96, 32, 288, 70
+    wl = tiny("alg1", s=s, B=p, K=kv_bar - p, steps=gen, p_dec=p, dtype="bf16", d=128, Hq=8, Hkv=2)
+    calls = [("prefill", t, p, -1) for t in range(0, kv_bar, p)]
+    t1 = kv_bar
+    while t1 < s:
+        calls.append(("evict", 0, 0, kv_bar - p))
+        calls.append(("prefill", t1, min(p, s - t1), -1))
+        t1 += p
+    n = kv_bar
+    for t in range(gen):
+        if n == kv_bar:
+            calls.append(("evict", 0, 0, kv_bar - p))
+            n -= p
+        calls.append(("decode", s + t, 1, -1))
+        n += 1
+    run_lockstep(wl, all_units(wl), calls=calls, growth=p, check_rows_every=3)
+
+
+# ------------------------------------------------------------------ API behaviour on the device
+def test_error_codes_and_state_tracking():
+    wl = tiny("errors", dtype="bf16", d=128)
+    cfg = make_config(wl)
+    cache = bm.BatchMaxCache(cfg)
+    inp = Inputs(wl, "cuda")
+    q, k, v = inp.block(0, 0, 48)
+    with pytest.raises(bm.BMError) as e:
+        cache.prefill_block(q, k, v, 5)                                  # pos0 must follow curr_id
+    assert e.value.code == 4
+    q2 = torch.randn(2, 49, wl.Hq, wl.d, device="cuda").to(wl.torch_dtype)
+    with pytest.raises(bm.BMError) as e:
+        cache.prefill_block(q2, q2[:, :, :wl.Hkv].contiguous(), q2[:, :, :wl.Hkv].contiguous(), 0)
+    assert e.value.code == 1                                             # I > block_max
+    with pytest.raises(bm.BMError) as e:
+        cache.evict(-3)
+    assert e.value.code == 1
+    cache.close()
+    # capacity: appending without eviction beyond cap
+    cache = bm.BatchMaxCache(cfg)
+    cache.prefill_block(q, k, v, 0, evict_to=wl.K)
+    q, k, v = inp.block(0, 48, 48)
+    with pytest.raises(bm.BMError) as e:
+        cache.prefill_block(q, k, v, 48, evict_to=-1)
+    assert e.value.code == 3
+    assert cache.length() == (wl.K, 47)                                  # failed call left the mirror alone
+    # sample ranges with unequal n cannot share a call
+    cache.prefill_block(q[:1], k[:1], v[:1], 48, evict_to=wl.K, sample0=0)
+    with pytest.raises(bm.BMError) as e:
+        cache.prefill_block(q, k, v, 48, evict_to=wl.K)
+    assert e.value.code == 4
+    cache.prefill_block(q[1:], k[1:], v[1:], 48, evict_to=wl.K, sample0=1)
+    assert cache.length(sample=0) == cache.length(sample=1) == (wl.K, 95)
+    assert cache.status() == 0
+    cache.close()
+
+
+def run_free(wl, host=False, micro=None):
+    """Whole schedule on the GPU only; returns final state and all outputs (for determinism / variants)."""
+    cfg = make_config(wl)
+    cache = bm.BatchMaxCache(cfg)
+    inp = Inputs(wl, "cuda")
+    outs = []
+    for kind, pos0, I, ev in schedule(wl):
+        q, k, v = inp.block(0, pos0, I)
+        if kind == "decode":
+            q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
+        if host:
+            qh, kh, vh = (t.cpu().pin_memory() for t in (q, k, v))
+            oh = torch.empty_like(qh).pin_memory()
+            if kind == "prefill":
+                cache.prefill_block_host(qh, kh, vh, pos0, oh, evict_to=ev)
+            else:
+                cache.decode_step_host(qh, kh, vh, oh, evict_to=ev)
+            torch.cuda.synchronize()
+            outs.append(oh.clone())
+        elif micro and kind == "prefill":
+            o = torch.empty_like(q)
+            for s0 in range(0, wl.b, micro):
+                cache.prefill_block(q[s0:s0 + micro], k[s0:s0 + micro], v[s0:s0 + micro], pos0, out=o[s0:s0 + micro],
+                                    evict_to=ev, sample0=s0)
+            outs.append(o.cpu())
+        elif micro:
+            o = torch.empty_like(q)
+            for s0 in range(0, wl.b, micro):
+                cache.decode_step(q[s0:s0 + micro], k[s0:s0 + micro], v[s0:s0 + micro], out=o[s0:s0 + micro],
+                                  evict_to=ev, sample0=s0)
+            outs.append(o.cpu())
+        else:
+            o = cache.prefill_block(q, k, v, pos0, evict_to=ev) if kind == "prefill" else \
+                cache.decode_step(q, k, v, evict_to=ev)
+            outs.append(o.cpu())
+    state = [cache.export(0, s, h, rows=True) for s in range(wl.b) for h in range(wl.Hkv)]
+    cache.close()
+    return outs, state
+
+
+def assert_same_run(a, b):
+    for x, y in zip(a[0], b[0]):
+        assert torch.equal(x, y)
+    for sa, sb in zip(a[1], b[1]):
+        for x, y in zip(sa, sb):
+            assert torch.equal(x, y)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_bitwise_reproducible_and_variants_agree(dtype, d):
+    wl = tiny("repro", b=4, dtype=dtype, d=d, Hq=8, Hkv=2, s=256, B=64, K=64, steps=5)
+    base = run_free(wl)
+    assert_same_run(base, run_free(wl))                 # run-to-run determinism (no float atomics)
+    assert_same_run(base, run_free(wl, host=True))      # host-fed entry points
+    assert_same_run(base, run_free(wl, micro=1))        # sample ranges: micro-batched calls
+
+
+def test_export_import_roundtrip_resumes_identically():
+    wl = tiny("ckpt", dtype="bf16", d=128, Hq=8, Hkv=2, s=192, B=64, K=48, steps=0)
+    cfg = make_config(wl)
+    inp = Inputs(wl, "cuda")
+    a = bm.BatchMaxCache(cfg)
+    for kind, pos0, I, ev in schedule(wl)[:2]:
+        a.prefill_block(*inp.block(0, pos0, I), pos0, evict_to=ev)
+    b = bm.BatchMaxCache(cfg)
+    for s in range(wl.b):
+        n, cur = a.length(sample=s)
+        b.set_len(n, cur, sample=s)
+        for h in range(wl.Hkv):
+            b.import_(*a.export(0, s, h, rows=True), sample=s, kv_head=h)
+    kind, pos0, I, ev = schedule(wl)[2]
+    q, k, v = inp.block(0, pos0, I)
+    oa, ob = a.prefill_block(q, k, v, pos0, evict_to=ev), b.prefill_block(q, k, v, pos0, evict_to=ev)
+    assert torch.equal(oa, ob)
+    for s in range(wl.b):
+        for h in range(wl.Hkv):
+            for x, y in zip(a.export(0, s, h, rows=True), b.export(0, s, h, rows=True)):
+                assert torch.equal(x, y)
+
+
+def test_batch_sized_by_the_allocator_fits_its_arena():
+    # allocator: batch = max fitting a budget; both arms (P&D, decode-only compression) live in arenas of that size
+    wl = WORKLOADS["cfg3"].with_(s=1024, B=256, K=128, steps=2)
+    budget = 64 * 2 ** 20
+    pd_cfg = make_config(wl, batch=1)
+    do_cfg = make_config(wl, batch=1, growth=wl.s + 1 - wl.K)
+    b_pd, b_do = bm.max_batch(pd_cfg, budget), bm.max_batch(do_cfg, budget)
+    assert b_pd / b_do == pytest.approx((wl.s + 1) / (wl.K + 1), rel=0.08)
+    for b, growth in ((b_pd, None), (b_do, wl.s + 1 - wl.K)):
+        w = wl.with_(b=b)
+        cfg = make_config(w, growth=growth, max_call_samples=16)
+        assert bm.arena_bytes(cfg) <= budget
+        arena = torch.empty(budget + 512, dtype=torch.uint8, device="cuda")
+        arena[budget:] = 0xA5                                            # canary behind the arena
+        cache = bm.BatchMaxCache(cfg, arena=arena[:budget])
+        inp = Inputs(w, "cuda")
+        for pos0 in range(0, w.s, w.B):
+            for s0 in range(0, b, 16):
+                ns = min(16, b - s0)
+                q, k, v = inp.block(0, pos0, w.B, s0, ns)
+                cache.prefill_block(q, k, v, pos0, evict_to=(w.K if growth is None else -1), sample0=s0)
+        if growth is not None:
+            for s0 in range(0, b, 16):
+                cache.evict(w.K, sample0=s0, nsamples=min(16, b - s0))
+        torch.cuda.synchronize()
+        assert cache.status() == 0
+        assert cache.length(sample=b - 1)[0] == w.K
+        assert bool((arena[budget:] == 0xA5).all())
+        ids, sw, _, _ = cache.export(0, b - 1, w.Hkv - 1)
+        assert np.all(np.diff(ids.numpy()) > 0) and float(sw.min()) >= 0
+        cache.close()
