@@ -130,6 +130,25 @@ bm_status_t bm_decode_step(bm_cache_t* cache, int32_t layer, int32_t sample0, in
 bm_status_t bm_evict(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples, int32_t target,
                      void* cuda_stream);
 
+/* ---- bm_prefill_block for callers that cannot provide scratch (the paper has no counterpart) ----
+ * Identical to bm_prefill_block in arguments, result and errors, but the per-call scratch (log-sum-exp of
+ * the query rows, column sums of the new pairs) is taken from a fixed 5 MiB array that is part of the
+ * library image on every GPU that loads it, instead of the workspace given to bm_cache_create.  It is
+ * meant for callers that must not allocate device memory themselves: a serving loop whose memory plan is
+ * frozen after start-up, a plug-in under a framework whose caching allocator owns the whole device, or a
+ * thread that may not issue allocating CUDA calls.  The call itself allocates and frees nothing.
+ *   Limits: nsamples * Hq * I <= 1,048,576 and nsamples * Hkv * I <= 262,144, else BM_ERR_CAPACITY
+ *   (nothing is enqueued).  cfg.device must be below 64.
+ *   First call on a device: resolves the array's device address (cudaGetSymbolAddress with that device
+ *   current).  Make that first call before starting any stream capture.
+ *   Sharing: all handles and all calls on a device use the same array, and it keeps the previous call's
+ *   contents.  Nothing in it has to start from zero (every entry a call reads is written by that call
+ *   first), but two calls that overlap on the GPU -- different streams, or different handles without
+ *   stream ordering -- race on it and corrupt each other's scores. */
+bm_status_t bm_prefill_block_static(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples,
+                                    const void* q, const void* k, const void* v, int32_t I, int32_t pos0,
+                                    void* out, int32_t evict_to, void* cuda_stream);
+
 /* ---- the same two passes fed from HOST memory (end-to-end use without device-side producers) ----
  * q/k/v/out are HOST pointers (pinned memory makes the copies asynchronous); `staging` is a DEVICE
  * buffer of at least bm_staging_bytes(cfg, nsamples, I) bytes.  The call copies q, k, v to the device,

@@ -44,6 +44,7 @@ SIGNATURES = {
     "bm_cache_create": (_i32, [_cfgp, _vp, _sz, _vp, _sz, _vp, C.POINTER(_vp)]),
     "bm_cache_destroy": (_i32, [_vp]),
     "bm_prefill_block": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _vp, _i32, _vp]),
+    "bm_prefill_block_static": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _vp, _i32, _vp]),
     "bm_decode_step": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp]),
     "bm_evict": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp]),
     "bm_staging_bytes": (_i32, [_cfgp, _i32, _i32, C.POINTER(_sz)]),
@@ -220,6 +221,18 @@ class BatchMaxCache:
             out = self.torch.empty_like(q)
         _check(lib().bm_prefill_block(self.h, layer, sample0, ns, _ptr(q), _ptr(k), _ptr(v), I, pos0, _ptr(out),
                                       evict_to, _stream(stream)), "bm_prefill_block")
+        return out
+
+    def prefill_block_static(self, q, k, v, pos0: int, out=None, evict_to: int = -1, layer: int = 0,
+                             sample0: int = 0, stream=None):
+        """bm_prefill_block_static: same pass, scratch taken from the array built into the library (for callers
+        that cannot allocate a workspace).  Size limits and sharing rules are in include/batchmax.h."""
+        ns, I = q.shape[0], q.shape[1]
+        assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and q.dtype == self.tdtype
+        if out is None:
+            out = self.torch.empty_like(q)
+        _check(lib().bm_prefill_block_static(self.h, layer, sample0, ns, _ptr(q), _ptr(k), _ptr(v), I, pos0,
+                                             _ptr(out), evict_to, _stream(stream)), "bm_prefill_block_static")
         return out
 
     def decode_step(self, q, k, v, out=None, evict_to: int = -1, layer: int = 0, sample0: int = 0, stream=None):

@@ -520,3 +520,47 @@ const char* bm_status_string(bm_status_t s) {
 }
 
 }  // extern "C"
+
+// ---- prefill block with library-resident scratch -------------------------------------------------------
+// Some callers cannot hand the library a workspace they allocated: a serving loop that froze its memory
+// plan at start-up, a plug-in running under a framework whose caching allocator owns all device memory,
+// or a host thread that is not allowed to make allocating CUDA calls at all.  For them the per-call
+// scratch of the block forward pass (the log-sum-exp of every query row and the new pairs' column sums)
+// lives in a fixed array inside the library image.  Every GPU that loads the library holds these
+// kStaticLseFloats + kStaticNewSumFloats floats (5 MiB) until the process exits.
+namespace {
+constexpr size_t kStaticLseFloats = 1u << 20;     // nsamples * Hq  * I  <= 1,048,576
+constexpr size_t kStaticNewSumFloats = 1u << 18;  // nsamples * Hkv * I  <=   262,144
+constexpr int kMaxDevices = 64;
+static __device__ __align__(256) float g_static_scratch[kStaticLseFloats + kStaticNewSumFloats];
+// Device address of g_static_scratch per device ordinal.  In host code the symbol itself is only a
+// stand-in, never a device address, so it is resolved once per device with that device current.
+float* g_static_scratch_addr[kMaxDevices] = {};
+}  // namespace
+
+extern "C" bm_status_t bm_prefill_block_static(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples,
+                                               const void* q, const void* k, const void* v, int32_t I,
+                                               int32_t pos0, void* out, int32_t evict_to, void* cuda_stream) {
+  if (c == nullptr) return BM_ERR_INVALID;
+  if (nsamples < 1 || I < 1) return BM_ERR_INVALID;
+  const int dev = c->cfg.device;
+  if (dev < 0 || dev >= kMaxDevices) return BM_ERR_INVALID;
+  if ((size_t)nsamples * c->cfg.n_q_heads * (size_t)I > kStaticLseFloats ||
+      (size_t)nsamples * c->cfg.n_kv_heads * (size_t)I > kStaticNewSumFloats)
+    return BM_ERR_CAPACITY;  // the call needs more scratch than the built-in array holds
+  if (g_static_scratch_addr[dev] == nullptr) {
+    if (cudaSetDevice(dev) != cudaSuccess) return BM_ERR_CUDA;
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return BM_ERR_CUDA;
+    g_static_scratch_addr[dev] = static_cast<float*>(p);
+  }
+  // Run the ordinary pass with the handle's scratch pointers redirected for the duration of the call.
+  float* const lse_saved = c->ws_lse;
+  float* const new_sum_saved = c->ws_new_sum;
+  c->ws_lse = g_static_scratch_addr[dev];
+  c->ws_new_sum = g_static_scratch_addr[dev] + kStaticLseFloats;
+  const bm_status_t s = bm_prefill_block(c, layer, sample0, nsamples, q, k, v, I, pos0, out, evict_to, cuda_stream);
+  c->ws_lse = lse_saved;
+  c->ws_new_sum = new_sum_saved;
+  return s;
+}
