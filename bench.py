@@ -40,8 +40,12 @@ def parse_args():
     ap.add_argument("--workload", default="cfg2")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="launch every call eagerly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
+    ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (roofline runs)")
+    ap.add_argument("--prompt", type=int, default=None, help="override the workload's prompt length")
+    ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
     return ap.parse_args()
 
 
@@ -67,6 +71,22 @@ def peaks():
         d = json.load(open(p))
         return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
     return dict(FALLBACK_PEAKS), "fallback"
+
+
+def max_over_ranks(x: float, device="cpu") -> float:
+    """Largest value of x over all ranks of the default process group (x itself without one)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Replicas: every rank pushes the same number of tokens per step; the job's step time is the slowest rank's."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
 class ClockSampler:
@@ -174,6 +194,9 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     from paper_2412_05693_b200.workloads import WORKLOADS
     wl = WORKLOADS[args.workload]
+    over = {k: v for k, v in (("b", args.batch), ("s", args.prompt), ("steps", args.decode_steps)) if v is not None}
+    if over:   # roofline runs: the named shape at another batch / prompt length (reported in `config`)
+        wl = wl.with_(name=wl.name + "+" + ",".join(f"{k}={v}" for k, v in over.items()), **over)
 
     if args.impl == "reference":
         if rank != 0:
@@ -220,8 +243,10 @@ def main():
     arena = torch.empty(bm.arena_bytes(cfg), dtype=torch.uint8, device=dev)
     flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device=dev)
 
+    workspace = torch.empty(max(bm.workspace_bytes(cfg), 256), dtype=torch.uint8, device=dev)
+
     def one_step(host_bufs=None):
-        cache = bm.BatchMaxCache(cfg, arena=arena)
+        cache = bm.BatchMaxCache(cfg, arena=arena, workspace=workspace)
         for layer in range(wl.L):
             for ci, (kind, pos0, I, ev) in enumerate(calls):
                 if host_bufs is None:
@@ -238,10 +263,19 @@ def main():
                         cache.decode_step_host(q, k, v, o, evict_to=ev, layer=layer)
         return cache
 
-    def timed(n_warm, n_steps, host_bufs=None):
+    def timed(n_warm, n_steps, host_bufs=None, use_graph=False):
         for _ in range(n_warm):
             one_step(host_bufs).close()
         torch.cuda.synchronize()
+        graph = None
+        if use_graph:
+            # every call of the step is stream-ordered and allocation-free, so the whole step (cache creation,
+            # all prefill blocks, all decode steps) is captured once and replayed
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                one_step(host_bufs).close()
+            graph.replay()
+            torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
@@ -250,28 +284,29 @@ def main():
             flush.fill_(1)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            c = one_step(host_bufs)
+            if graph is not None:
+                graph.replay()
+            else:
+                one_step(host_bufs).close()
             e1.record(stream)
             e1.synchronize()
-            c.close()
             ms.append(e0.elapsed_time(e1))
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
-        total = torch.tensor([sum(ms)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(total, op=dist.ReduceOp.MAX)
-        return float(total.item()) / n_steps
+        return max_over_ranks(sum(ms), dev) / n_steps
 
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
     launches0 = bm.kernel_launch_count()
-    ms_step = timed(args.warmup, args.steps)
-    launches = (bm.kernel_launch_count() - launches0) // (args.warmup + args.steps) * args.steps
+    one_step().close()
+    launches_per_step = bm.kernel_launch_count() - launches0
+    ms_step = timed(args.warmup, args.steps, use_graph=not args.no_graph)
+    launches = launches_per_step * args.steps
     clocks = sampler.stop() if rank == 0 else None
     tokens = workload_tokens(wl)
-    value = world * tokens / (ms_step * 1e-3)
+    value = whole_job_value(tokens, world, ms_step)
 
     # ---- dominant kernel: the prefill-block attention forward, timed per launch with CUDA events
     prof = bm.binding.profile_pass(lambda: one_step().close()) if hasattr(bm.binding, "profile_pass") else None
@@ -312,7 +347,7 @@ def main():
             h2d += sum(t.numel() * t.element_size() for t in (hq, hk, hv))
             d2h += ho.numel() * ho.element_size()
         ms_e2e = timed(1, max(1, min(args.steps, 3)), host_bufs)
-        e2e = {"value": world * tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d * wl.L,
+        e2e = {"value": whole_job_value(tokens, world, ms_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d * wl.L,
                "d2h_bytes_per_step": d2h * wl.L, "ms_per_step": ms_e2e}
         del host_bufs
 
@@ -329,7 +364,8 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
                 "config": cfg_dict(wl, {"parallelism": f"replicas x{world}" if world > 1 else "single GPU",
-                                        "prefill_path": "tcgen05" if bm.last_prefill_path() == 1 else "simt-fp32"}),
+                                        "prefill_path": "tcgen05" if bm.last_prefill_path() == 1 else "simt-fp32",
+                                        "launch": "eager" if args.no_graph else "one CUDA graph per step, replayed"}),
                 "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
                 "clocks": clocks, "prefill_useful_tflop_per_step": 4.0 * wl.d * ppairs / 1e12}
         line.update(extra)

@@ -183,14 +183,15 @@ def _stream(stream):
 class BatchMaxCache:
     """Handle of one bm_cache_t plus the torch tensors backing its arena and workspace."""
 
-    def __init__(self, cfg: Config, arena=None, stream=None):
+    def __init__(self, cfg: Config, arena=None, stream=None, workspace=None):
         import torch
         self.cfg = cfg
         self.torch = torch
         dev = torch.device("cuda", cfg.device)
         need = arena_bytes(cfg)
         self.arena = arena if arena is not None else torch.empty(need, dtype=torch.uint8, device=dev)
-        self.workspace = torch.empty(max(workspace_bytes(cfg), 256), dtype=torch.uint8, device=dev)
+        self.workspace = workspace if workspace is not None else \
+            torch.empty(max(workspace_bytes(cfg), 256), dtype=torch.uint8, device=dev)
         self.tdtype = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
         self._staging = None
         h = _vp(None)

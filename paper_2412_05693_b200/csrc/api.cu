@@ -285,22 +285,21 @@ bm_status_t bm_decode_step(bm_cache_t* c, int32_t layer, int32_t sample0, int32_
   const int n1 = n_old + 1;
   if (n1 > c->cap) return BM_ERR_CAPACITY;
   const int target = (evict_to >= 0 && n1 > evict_to) ? evict_to : -1;
-  if (n1 > kMaxCandidates || decode_smem_bytes(c->cfg.head_dim, c->g, n1, target) > kMaxSmem) return BM_ERR_CAPACITY;
+  const bool mma = c->cfg.dtype == BM_BF16;   // bf16 caches decode on the tensor-core kernel, fp32 caches on the SIMT one
+  const size_t smem = mma ? decode_mma_smem_bytes(c->cfg.head_dim, c->g, n1, target)
+                          : decode_smem_bytes(c->cfg.head_dim, c->g, n1, target);
+  if (n1 > kMaxCandidates || smem > kMaxSmem) return BM_ERR_CAPACITY;
   if ((s = set_device(c)) != BM_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   CacheView view = make_view(c, layer, sample0, nsamples, n_old);
   const int pos = curr + 1;
-  int n_new = n1;
-  if (target == 0) {
-    // nothing survives: run the attention and the update, then empty the caches on the host mirror
-    if (launch_decode(c->cfg.dtype, c->cfg.head_dim, view, q, k, v, out, pos, c->scale, -1, st) != cudaSuccess)
-      return BM_ERR_CUDA;
-    n_new = 0;
-  } else {
-    if (launch_decode(c->cfg.dtype, c->cfg.head_dim, view, q, k, v, out, pos, c->scale, target, st) != cudaSuccess)
-      return BM_ERR_CUDA;
-    if (target > 0) n_new = target;
-  }
+  // target 0: nothing survives -- run the attention and the update, then empty the caches on the host mirror
+  const int kernel_target = target == 0 ? -1 : target;
+  const cudaError_t err = mma ? launch_decode_mma(c->cfg.head_dim, view, q, k, v, out, pos, c->scale, kernel_target, st)
+                              : launch_decode(c->cfg.dtype, c->cfg.head_dim, view, q, k, v, out, pos, c->scale,
+                                              kernel_target, st);
+  if (err != cudaSuccess) return BM_ERR_CUDA;
+  const int n_new = target >= 0 ? target : n1;
   set_mirror(c, layer, sample0, nsamples, n_new, pos);
   return BM_OK;
 }

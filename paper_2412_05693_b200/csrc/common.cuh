@@ -49,6 +49,9 @@ cudaError_t launch_score_simt(int dtype, int d, const CacheView& c, const BlockA
 cudaError_t launch_evict(int dtype, int d, const CacheView& c, const EvictArgs& e, cudaStream_t st);
 cudaError_t launch_decode(int dtype, int d, const CacheView& c, const void* q, const void* k, const void* v,
                           void* out, int32_t pos, float scale, int32_t target /* <0: none */, cudaStream_t st);
+cudaError_t launch_decode_mma(int d, const CacheView& c, const void* q, const void* k, const void* v, void* out,
+                              int32_t pos, float scale, int32_t target /* <0: none */, cudaStream_t st);
+size_t decode_mma_smem_bytes(int d, int g, int n_rows, int target);
 size_t evict_smem_bytes(int n_cand, int target);
 size_t decode_smem_bytes(int d, int g, int n_rows, int target);
 bool tc_path_available();

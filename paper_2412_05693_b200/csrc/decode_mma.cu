@@ -1,0 +1,386 @@
+// bf16 decoding step (Algorithm 1 "generate token", Sec. 3.2 with I = 1), one CTA per (sample, kv-head) cache.
+// Same steps as the fp32 kernel in decode.cu, but the two contractions run on warp-level tensor-core MMAs
+// (m16n8k16, bf16 in, fp32 accumulate) fed straight from 128-bit global loads, so that the kernel issues few
+// enough instructions to be limited by HBM bandwidth:
+//   logits^T [16 keys x heads] = K-tile [16 keys x d] . q^T          (heads padded to 8 columns)
+//   out^T    [16 d    x heads] = V-tile^T [16 d x 16 keys] . p^T
+// Both contractions are invariant under a permutation of the contracted index, and the output index of the
+// second one can be un-permuted when it is written, so every thread loads whole 16-byte pieces of cache
+// rows (coalesced) and the MMA fragment slots are assigned to whatever elements those loads delivered.
+#include "evict.cuh"
+
+namespace bm {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kRowsPerIter = kWarps * 16;   // one 16-key tile per warp and iteration
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct DecodeArgs {
+  const void* q;
+  const void* k;
+  const void* v;
+  void* out;
+  int32_t pos;
+  float scale;
+  int32_t target;
+};
+
+struct Smem {
+  float* p;       // [G][n1t]  logits, then probabilities (zero beyond n1)
+  float* score;   // [n1t]
+  int32_t* id;    // [n1t]
+  float* wred;    // [2][G][warps]
+  float* best;    // [2][warps]
+  float* ored;    // [warps][G][D]
+};
+
+__host__ __device__ inline size_t smem_layout(unsigned char* base, int d, int g, int n1, Smem* s) {
+  const size_t n1t = (size_t)((n1 + 15) & ~15);
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) & ~size_t(15); return o; };
+  const size_t op = take(4 * (size_t)g * n1t), os = take(4 * n1t), oi = take(4 * n1t);
+  const size_t ow = take(4 * 2 * (size_t)g * kWarps), ob = take(4 * 2 * kWarps), oo = take(4 * (size_t)kWarps * g * d);
+  if (s != nullptr) {
+    s->p = reinterpret_cast<float*>(base + op);
+    s->score = reinterpret_cast<float*>(base + os);
+    s->id = reinterpret_cast<int32_t*>(base + oi);
+    s->wred = reinterpret_cast<float*>(base + ow);
+    s->best = reinterpret_cast<float*>(base + ob);
+    s->ored = reinterpret_cast<float*>(base + oo);
+  }
+  return off;
+}
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t r;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+  return r;
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint4 ldg16_or_zero(const __nv_bfloat16* p, bool ok) {
+  return ok ? ld_global_16(p) : make_uint4(0u, 0u, 0u, 0u);
+}
+
+template <int D, int G>
+__global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, DecodeArgs a) {
+  using T = __nv_bfloat16;
+  constexpr int QR = D / 32;   // 32-element rounds of the logits contraction
+  constexpr int VR = D / 64;   // 64-element rounds of the output contraction
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int n1 = c.n_old + 1;
+  const int n1t = (n1 + 15) & ~15;
+  Smem s;
+  smem_layout(smem_raw, D, G, n1, &s);
+
+  const int unit = blockIdx.x, smp = unit / c.Hkv, kh = unit % c.Hkv;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gid = lane >> 2, tq = lane & 3;   // MMA fragment coordinates: group id, thread in group
+  const size_t base = (size_t)unit * c.cap;
+  T* kslab = reinterpret_cast<T*>(c.k_slab) + base * D;
+  T* vslab = reinterpret_cast<T*>(c.v_slab) + base * D;
+  const bool evict_one = (a.target == n1 - 1);
+  const bool evict_general = (a.target >= 0 && a.target < n1 - 1);
+
+  // the step's pair -> row n_old of the cache; ids -> smem
+  if (tid < 2 * (D / 8)) {
+    const int pc = tid % (D / 8);
+    const T* src = reinterpret_cast<const T*>(tid < D / 8 ? a.k : a.v) + ((size_t)smp * c.Hkv + kh) * D + pc * 8;
+    T* dst = (tid < D / 8 ? kslab : vslab) + (size_t)c.n_old * D + pc * 8;
+    st_global_16(dst, ld_global_16(src));
+  }
+  for (int j = tid; j < n1t; j += kThreads) s.id[j] = (j < c.n_old) ? c.kv_ids[base + j] : a.pos;
+  // q fragments: thread (gid, tq) holds, for every 32-element round, the 8 elements [32r + 8tq, +8) of head gid
+  uint32_t qf[QR][4];
+  {
+    const T* qp = reinterpret_cast<const T*>(a.q) + ((size_t)smp * c.Hq + kh * G + gid) * D;
+#pragma unroll
+    for (int r = 0; r < QR; ++r) {
+      const uint4 w = ldg16_or_zero(qp + 32 * r + 8 * tq, gid < G);
+      qf[r][0] = w.x; qf[r][1] = w.y; qf[r][2] = w.z; qf[r][3] = w.w;
+    }
+  }
+  __syncthreads();
+
+  const float sc2 = a.scale * kLog2e;
+  const int n_iter = (n1 + kRowsPerIter - 1) / kRowsPerIter;   // same trip count for every thread
+
+  // ---- logits (log2 domain).  Tile rows gid and gid+8; the k-slots of thread tq are its own 8 elements.
+  for (int it = 0; it < n_iter; ++it) {
+    const int tb = it * kRowsPerIter + warp * 16;
+    const int j0 = tb + gid, j1 = tb + gid + 8;
+    uint4 x[QR], y[QR];
+#pragma unroll
+    for (int r = 0; r < QR; ++r) {
+      x[r] = ldg16_or_zero(kslab + (size_t)j0 * D + 32 * r + 8 * tq, j0 < n1);
+      y[r] = ldg16_or_zero(kslab + (size_t)j1 * D + 32 * r + 8 * tq, j1 < n1);
+    }
+    float cacc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int r = 0; r < QR; ++r) {
+      mma16816(cacc, x[r].x, y[r].x, x[r].y, y[r].y, qf[r][0], qf[r][1]);
+      mma16816(cacc, x[r].z, y[r].z, x[r].w, y[r].w, qf[r][2], qf[r][3]);
+    }
+    // cacc[0], cacc[1]: key j0, heads 2tq, 2tq+1 ; cacc[2], cacc[3]: key j1
+    if (2 * tq < G) {
+      if (j0 < n1) s.p[(2 * tq) * n1t + j0] = cacc[0] * sc2;
+      if (j1 < n1) s.p[(2 * tq) * n1t + j1] = cacc[2] * sc2;
+    }
+    if (2 * tq + 1 < G) {
+      if (j0 < n1) s.p[(2 * tq + 1) * n1t + j0] = cacc[1] * sc2;
+      if (j1 < n1) s.p[(2 * tq + 1) * n1t + j1] = cacc[3] * sc2;
+    }
+  }
+  __syncthreads();
+
+  // ---- softmax over the n1 rows, per head
+  float inv[G];
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    float m = -INFINITY;
+    for (int j = tid; j < n1; j += kThreads) m = fmaxf(m, s.p[h * n1t + j]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    if (lane == 0) s.wred[h * kWarps + warp] = m;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    float m = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) m = fmaxf(m, s.wred[h * kWarps + w]);
+    float t = 0.f;
+    for (int j = tid; j < n1; j += kThreads) {
+      const float e = ex2f(s.p[h * n1t + j] - m);
+      s.p[h * n1t + j] = e;
+      t += e;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+    if (lane == 0) s.wred[(G + h) * kWarps + warp] = t;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int h = 0; h < G; ++h) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) t += s.wred[(G + h) * kWarps + w];  // fixed order
+    inv[h] = 1.f / t;
+  }
+
+  // ---- normalise, sum_weights += attn_weights (heads added in a fixed order), candidate for eviction
+  float best_ave = INFINITY;
+  int best_j = -1;
+  for (int j = tid; j < n1t; j += kThreads) {
+    if (j >= n1) {
+#pragma unroll
+      for (int h = 0; h < G; ++h) s.p[h * n1t + j] = 0.f;   // padding keys carry no weight
+      continue;
+    }
+    float add = 0.f;
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      const float p = s.p[h * n1t + j] * inv[h];
+      s.p[h * n1t + j] = p;
+      add += p;
+    }
+    const float sw = ((j < c.n_old) ? c.sum_weights[base + j] : 0.f) + add;
+    s.score[j] = sw;
+    if (evict_one) {
+      const float ave = sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
+      if (ave <= best_ave) { best_ave = ave; best_j = j; }   // j ascends: ties move to the higher position
+    } else {
+      c.sum_weights[base + j] = sw;
+    }
+  }
+  int hole = n1;  // no row leaves
+  if (evict_one) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      const float oa = __shfl_xor_sync(0xffffffffu, best_ave, off);
+      const int oj = __shfl_xor_sync(0xffffffffu, best_j, off);
+      if (oa < best_ave || (oa == best_ave && oj > best_j)) { best_ave = oa; best_j = oj; }
+    }
+    if (lane == 0) { s.best[warp] = best_ave; reinterpret_cast<int*>(s.best)[kWarps + warp] = best_j; }
+    __syncthreads();
+    best_ave = s.best[0];
+    best_j = reinterpret_cast<int*>(s.best)[kWarps];
+#pragma unroll
+    for (int w = 1; w < kWarps; ++w) {
+      const float oa = s.best[w];
+      const int oj = reinterpret_cast<int*>(s.best)[kWarps + w];
+      if (oa < best_ave || (oa == best_ave && oj > best_j)) { best_ave = oa; best_j = oj; }
+    }
+    hole = best_j;
+    // sum_weights / kv_ids in their final places: rows behind the hole move up by one
+    for (int j = tid; j < n1; j += kThreads) {
+      if (j < hole) c.sum_weights[base + j] = s.score[j];
+      else if (j > hole) { c.sum_weights[base + j - 1] = s.score[j]; c.kv_ids[base + j - 1] = s.id[j]; }
+    }
+  } else {
+    if (tid == 0) c.kv_ids[base + c.n_old] = a.pos;
+    __syncthreads();
+  }
+
+  // ---- out^T = V^T p^T.  Thread (gid, tq) loads, from the 4 rows tb + 4tq + {0..3}, the 8 elements
+  // [64r + 8gid, +8); MMA m uses element m as fragment row gid and element m+4 as row gid+8.
+  float oacc[VR][4][4];
+#pragma unroll
+  for (int r = 0; r < VR; ++r)
+#pragma unroll
+    for (int m = 0; m < 4; ++m)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) oacc[r][m][e] = 0.f;
+  for (int it = 0; it < n_iter; ++it) {
+    const int tb = it * kRowsPerIter + warp * 16;
+    const int jr = tb + 4 * tq;   // first of this thread's 4 rows
+    uint4 z[VR][4];
+#pragma unroll
+    for (int r = 0; r < VR; ++r)
+#pragma unroll
+      for (int sx = 0; sx < 4; ++sx)
+        z[r][sx] = ldg16_or_zero(vslab + (size_t)(jr + sx) * D + 64 * r + 8 * gid, jr + sx < n1);
+    // p^T fragment: (head gid; keys jr, jr+1) and (head gid; keys jr+2, jr+3)
+    uint32_t pb0 = 0u, pb1 = 0u;
+    if (gid < G && jr < n1t) {
+      const float4 pv = *reinterpret_cast<const float4*>(&s.p[gid * n1t + jr]);
+      pb0 = pack2(pv.x, pv.y);
+      pb1 = pack2(pv.z, pv.w);
+    }
+#pragma unroll
+    for (int r = 0; r < VR; ++r) {
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        // element m of the 8 loaded: 32-bit word m/2, half m%2 ; element m+4: word 2 + m/2, same half
+        const uint32_t sel = (m & 1) ? 0x7632u : 0x5410u;
+        const uint32_t w0 = (m < 2) ? z[r][0].x : z[r][0].y, w1 = (m < 2) ? z[r][1].x : z[r][1].y;
+        const uint32_t w2 = (m < 2) ? z[r][2].x : z[r][2].y, w3 = (m < 2) ? z[r][3].x : z[r][3].y;
+        const uint32_t u0 = (m < 2) ? z[r][0].z : z[r][0].w, u1 = (m < 2) ? z[r][1].z : z[r][1].w;
+        const uint32_t u2 = (m < 2) ? z[r][2].z : z[r][2].w, u3 = (m < 2) ? z[r][3].z : z[r][3].w;
+        mma16816(oacc[r][m], prmt(w0, w1, sel), prmt(u0, u1, sel), prmt(w2, w3, sel), prmt(u2, u3, sel), pb0, pb1);
+      }
+    }
+    if (evict_one && (it + 1) * kRowsPerIter > hole) {   // uniform over the CTA
+      __syncthreads();                                   // every load of rows < (it+1)*kRowsPerIter has completed
+#pragma unroll
+      for (int r = 0; r < VR; ++r)
+#pragma unroll
+        for (int sx = 0; sx < 4; ++sx) {
+          const int j = jr + sx;
+          if (j < n1 && j > hole) st_global_16(vslab + (size_t)(j - 1) * D + 64 * r + 8 * gid, z[r][sx]);
+        }
+    }
+  }
+  // K rows behind the hole: one-row shift (re-read, mostly from L2: the logits pass just streamed them)
+  if (evict_one) {
+    constexpr int PR = D / 8;                 // 16-byte pieces per row
+    constexpr int RPI = kThreads / PR * 4;    // rows per iteration, 4 pieces per thread
+    const int slot = tid / PR, pc = tid % PR;
+    for (int r0 = (hole / RPI) * RPI; r0 < n1; r0 += RPI) {
+      uint4 raw[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j = r0 + slot + u * (kThreads / PR);
+        if (j < n1 && j > hole) raw[u] = ld_global_16(kslab + (size_t)j * D + pc * 8);
+      }
+      __syncthreads();
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j = r0 + slot + u * (kThreads / PR);
+        if (j < n1 && j > hole) st_global_16(kslab + (size_t)(j - 1) * D + pc * 8, raw[u]);
+      }
+    }
+  }
+
+  // ---- combine the warps' partial outputs in a fixed order.  oacc[r][m][0..1]: element 64r + 8gid + m of heads
+  // 2tq, 2tq+1; oacc[r][m][2..3]: element 64r + 8gid + m + 4.
+#pragma unroll
+  for (int r = 0; r < VR; ++r)
+#pragma unroll
+    for (int m = 0; m < 4; ++m)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int h = 2 * tq + (e & 1);
+        const int dd = 64 * r + 8 * gid + m + ((e & 2) ? 4 : 0);
+        if (h < G) s.ored[(warp * G + h) * D + dd] = oacc[r][m][e];
+      }
+  __syncthreads();
+  for (int t = tid; t < G * D; t += kThreads) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) tot += s.ored[w * G * D + t];
+    T* op = reinterpret_cast<T*>(a.out) + ((size_t)smp * c.Hq + kh * G) * D;
+    op[t] = __float2bfloat16_rn(tot);
+  }
+
+  if (evict_general) {
+    __syncthreads();
+    CacheView cv = c;
+    cv.n_old = n1;
+    EvictArgs e;
+    e.blk_k = nullptr; e.blk_v = nullptr; e.new_sum = nullptr;
+    e.I = 0; e.pos0 = 0; e.curr_id = a.pos; e.target = a.target;
+    evict_body<T, D, kThreads>(cv, unit, smp, kh, e, smem_raw);
+  }
+}
+
+template <int D, int G>
+cudaError_t launch_t(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
+  const size_t smem = decode_mma_smem_bytes(D, G, c.n_old + 1, a.target);
+  static size_t configured = 0;
+  if (smem > configured) {
+    cudaError_t err = cudaFuncSetAttribute(decode_mma_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    configured = smem;
+  }
+  ProfileScope prof(kDecode, st);
+  decode_mma_kernel<D, G><<<c.nsamples * c.Hkv, kThreads, smem, st>>>(c, a);
+  count_launch();
+  return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t launch_g(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
+  switch (c.g) {
+    case 1: return launch_t<D, 1>(c, a, st);
+    case 2: return launch_t<D, 2>(c, a, st);
+    case 4: return launch_t<D, 4>(c, a, st);
+    case 8: return launch_t<D, 8>(c, a, st);
+    default: return cudaErrorInvalidValue;
+  }
+}
+
+}  // namespace
+
+size_t decode_mma_smem_bytes(int d, int g, int n_rows, int target) {
+  const size_t attn = smem_layout(nullptr, d, g, n_rows, nullptr);
+  const size_t ev = (target >= 0 && target < n_rows - 1) ? evict_smem_bytes(n_rows, target) : 0;
+  return attn > ev ? attn : ev;
+}
+
+cudaError_t launch_decode_mma(int d, const CacheView& c, const void* q, const void* k, const void* v, void* out,
+                              int32_t pos, float scale, int32_t target, cudaStream_t st) {
+  DecodeArgs a{q, k, v, out, pos, scale, target};
+  if (d == 64) return launch_g<64>(c, a, st);
+  if (d == 128) return launch_g<128>(c, a, st);
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace bm
