@@ -1,13 +1,14 @@
 // bf16 tensor-core path of the block forward pass (Sec. 3.2) for sm_100a:
 //   attn_fwd_tc : out = softmax(scale q k^T) v over the cached pairs and the block's causal pairs, plus the
-//                 log2-sum-exp of every query row.  QK^T and PV run on tcgen05 with TMA-staged tiles and
-//                 TMEM accumulators; a warp-specialised CTA (TMA producer / MMA issuer / 4 softmax warps)
-//                 handles one tile of 128 query rows.
+//                 log2-sum-exp of every query row.  QK^T and PV run on tcgen05 with TMA-staged tiles and TMEM
+//                 accumulators.  One CTA owns two tiles of 128 query rows of the same (sample, kv-head) unit;
+//                 two softmax warpgroups work on them alternately so that one tile's exponentials overlap the
+//                 other tile's MMAs, and both tiles share every K/V tile that is loaded.
 //   score_tc    : sum_weights += sum_i attn_weights[i].  Recomputes the transposed logits S^T = K Q^T so that
 //                 a TMEM lane is a key; each thread then sums exp2(s - lse) over the queries of its own key
 //                 in a fixed order (deterministic, no atomics).
-// Query rows of a (sample, kv-head) unit are ordered r = i * g + h (input i, head h of the group), so one
-// tile of 128 rows shares every K/V tile it loads among the g heads of the group.
+// Query rows of a unit are ordered r = i * g + h (input i, head h of the group), so a tile of 128 rows shares
+// its K/V tiles among the g heads of the group.
 #include "tc_common.cuh"
 #include "common.cuh"
 
@@ -16,16 +17,14 @@ namespace {
 
 using namespace tc;
 
-constexpr int kTileM = 128;      // query rows per CTA tile
+constexpr int kTileM = 128;      // query rows per tile
 constexpr int kTileN = 128;      // keys per tile
-constexpr int kFwdThreads = 192; // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: softmax / epilogue
-constexpr int kStages = 2;       // K/V ring depth
-constexpr int kTmemCols = 512;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;  // stale row max is kept until the true max exceeds it by 2^8
 
 struct TcMaps {
   CUtensorMap q;       // 5-d: (d, g, Hkv, I, nsamples)
+  CUtensorMap o;       // same shape over the output
   CUtensorMap k_slab;  // 3-d: (d, n_old, units)
   CUtensorMap v_slab;
   CUtensorMap k_blk;   // 4-d: (d, Hkv, I, nsamples)
@@ -35,7 +34,6 @@ struct TcMaps {
 struct TcArgs {
   int n_old, I, g, Hq, Hkv;
   float scale_log2;  // softmax scale * log2(e)
-  void* out;
   float* lse2;       // [units][I*g] log2-sum-exp (log2 domain, scaled logits)
   float* sum_weights;
   float* new_sum;
@@ -43,22 +41,26 @@ struct TcArgs {
   int* status;
 };
 
+// ------------------------------------------------------------------------------------------------------
+// Forward.  Warps 0-3: softmax of tile A, warps 4-7: softmax of tile B, warp 8: MMA issue + TMEM owner,
+// warp 9: TMA producer.  TMEM: S_A | S_B (fp32 logits, overwritten in place by the bf16 probabilities that
+// feed P.V as the tensor-memory operand) | O_A | O_B.
+constexpr int kFwdThreads = 320;
+constexpr int kKvStages = 4;     // ring of K/V tiles: entry 2j = K_j, entry 2j+1 = V_j
+constexpr int kTmemCols = 512;
+
 template <int D>
 struct FwdSmem {
   static constexpr int kChunks = D / 64;                 // 64-element (128-byte) column chunks per row
   static constexpr int kTileBytes = kChunks * 16384;     // 128 rows x D bf16
-  static constexpr int kQ = 0;
-  static constexpr int kK = kQ + kTileBytes;
-  static constexpr int kV = kK + kStages * kTileBytes;
-  static constexpr int kP = kV + kStages * kTileBytes;   // 128 x 128 bf16 probabilities
-  static constexpr int kBars = kP + 2 * 16384;
+  static constexpr int kQ = 0;                           // two query tiles (reused to stage the outputs)
+  static constexpr int kKV = kQ + 2 * kTileBytes;
+  static constexpr int kBars = kKV + kKvStages * kTileBytes;
   static constexpr int kTotal = kBars + 256 + 1024;      // + barriers + alignment slack
 };
 
-// barrier indices
-enum { B_QFULL = 0, B_KFULL = 1, B_VFULL = B_KFULL + kStages, B_KVEMPTY = B_VFULL + kStages,
-       B_SFULL = B_KVEMPTY + kStages, B_SFREE = B_SFULL + 2, B_PFULL = B_SFREE + 2, B_PVDONE = B_PFULL + 1,
-       B_COUNT = B_PVDONE + 1 };
+enum { B_QFULL = 0, B_KVFULL = 2, B_KVEMPTY = B_KVFULL + kKvStages, B_SFULL = B_KVEMPTY + kKvStages,
+       B_PFULL = B_SFULL + 2, B_ODONE = B_PFULL + 2, B_COUNT = B_ODONE + 2 };
 
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
@@ -73,181 +75,187 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int unit = blockIdx.y, smp = unit / a.Hkv, kh = unit % a.Hkv;
   const int R = a.I * a.g;
-  const int row0 = blockIdx.x * kTileM;
   const int qpt = kTileM / a.g;                  // inputs (positions) covered by one row tile
-  const int i0 = blockIdx.x * qpt;
-  const int i_last = min(a.I - 1, i0 + qpt - 1);
   const int t_old = (a.n_old + kTileN - 1) / kTileN;
-  const int t_new = i_last / kTileN + 1;
-  const int T = t_old + t_new;
+  int row0[2], i0[2], T[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) {
+    row0[x] = (blockIdx.x * 2 + x) * kTileM;
+    i0[x] = (blockIdx.x * 2 + x) * qpt;
+    const int i_last = min(a.I - 1, i0[x] + qpt - 1);
+    T[x] = t_old + i_last / kTileN + 1;          // cached-key tiles + block-key tiles up to the tile's last input
+  }
+  const bool active_b = row0[1] < R;
+  if (!active_b) T[1] = 0;
+  const int t_max = active_b ? T[1] : T[0];      // tile B sees at least as many key tiles as tile A
 
   if (tid == 0) {
     *abort_flag = 0;
-    mbar_init(&bars[B_QFULL], 1);
-    for (int s = 0; s < kStages; ++s) { mbar_init(&bars[B_KFULL + s], 1); mbar_init(&bars[B_VFULL + s], 1); mbar_init(&bars[B_KVEMPTY + s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&bars[B_SFULL + b], 1); mbar_init(&bars[B_SFREE + b], 128); }
-    mbar_init(&bars[B_PFULL], 128);
-    mbar_init(&bars[B_PVDONE], 1);
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(&bars[B_QFULL + x], 1);
+      mbar_init(&bars[B_SFULL + x], 1);
+      mbar_init(&bars[B_PFULL + x], 128);
+      mbar_init(&bars[B_ODONE + x], 1);
+    }
+    for (int s = 0; s < kKvStages; ++s) { mbar_init(&bars[B_KVFULL + s], 1); mbar_init(&bars[B_KVEMPTY + s], 1); }
     mbar_fence_init();
   }
-  if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+  if (warp == 8) tmem_alloc(tmem_slot, kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tm_s[2] = {tmem, tmem + 128};
-  const uint32_t tm_o = tmem + 256;
+  const uint32_t tm_o[2] = {tmem + 256, tmem + 384};
 
-  if (warp == 0) {
+  if (warp == 9) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      mbar_expect_tx(&bars[B_QFULL], L::kTileBytes);
-      for (int c = 0; c < L::kChunks; ++c)
-        tma_load_5d(sm + L::kQ + c * 16384, &maps.q, c * 64, 0, kh, i0, smp, &bars[B_QFULL]);
-      for (int j = 0; j < T; ++j) {
-        const int s = j % kStages;
-        if (j >= kStages) mbar_wait(&bars[B_KVEMPTY + s], ((j / kStages) - 1) & 1, abort_flag, a.status);
-        unsigned char* kd = sm + L::kK + s * L::kTileBytes;
-        unsigned char* vd = sm + L::kV + s * L::kTileBytes;
-        mbar_expect_tx(&bars[B_KFULL + s], L::kTileBytes);
+      for (int x = 0; x < (active_b ? 2 : 1); ++x) {
+        mbar_expect_tx(&bars[B_QFULL + x], L::kTileBytes);
+        for (int c = 0; c < L::kChunks; ++c)
+          tma_load_5d(sm + L::kQ + x * L::kTileBytes + c * 16384, &maps.q, c * 64, 0, kh, i0[x], smp, &bars[B_QFULL + x]);
+      }
+      for (int e = 0; e < 2 * t_max; ++e) {
+        const int j = e >> 1, s = e % kKvStages;
+        const bool is_v = e & 1;
+        if (e >= kKvStages) mbar_wait(&bars[B_KVEMPTY + s], ((e / kKvStages) - 1) & 1, abort_flag, a.status);
+        unsigned char* dst = sm + L::kKV + s * L::kTileBytes;
+        mbar_expect_tx(&bars[B_KVFULL + s], L::kTileBytes);
         for (int c = 0; c < L::kChunks; ++c) {
-          if (j < t_old) tma_load_3d(kd + c * 16384, &maps.k_slab, c * 64, j * kTileN, unit, &bars[B_KFULL + s]);
-          else tma_load_4d(kd + c * 16384, &maps.k_blk, c * 64, kh, (j - t_old) * kTileN, smp, &bars[B_KFULL + s]);
-        }
-        mbar_expect_tx(&bars[B_VFULL + s], L::kTileBytes);
-        for (int c = 0; c < L::kChunks; ++c) {
-          if (j < t_old) tma_load_3d(vd + c * 16384, &maps.v_slab, c * 64, j * kTileN, unit, &bars[B_VFULL + s]);
-          else tma_load_4d(vd + c * 16384, &maps.v_blk, c * 64, kh, (j - t_old) * kTileN, smp, &bars[B_VFULL + s]);
+          if (j < t_old)
+            tma_load_3d(dst + c * 16384, is_v ? &maps.v_slab : &maps.k_slab, c * 64, j * kTileN, unit, &bars[B_KVFULL + s]);
+          else
+            tma_load_4d(dst + c * 16384, is_v ? &maps.v_blk : &maps.k_blk, c * 64, kh, (j - t_old) * kTileN, smp,
+                        &bars[B_KVFULL + s]);
         }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 8) {
     // ------------------------------------------------------------------ MMA issuer (one thread)
     if (lane == 0) {
       const uint32_t idesc_qk = instr_desc(kTileM, kTileN, 0, 0);
       const uint32_t idesc_pv = instr_desc(kTileM, D, 0, 1);  // V is MN-major: d contiguous, keys along K
-      const uint32_t q_addr = smem_u32(sm + L::kQ), p_addr = smem_u32(sm + L::kP);
-      auto issue_pv = [&](int i) {
-        const int s = i % kStages;
-        mbar_wait(&bars[B_VFULL + s], (i / kStages) & 1, abort_flag, a.status);
-        mbar_wait(&bars[B_PFULL], i & 1, abort_flag, a.status);
-        tc_fence_after();
-        const uint32_t v_addr = smem_u32(sm + L::kV + s * L::kTileBytes);
-#pragma unroll
-        for (int ks = 0; ks < kTileN / 16; ++ks) {
-          const uint64_t da = smem_desc(p_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
-          const uint64_t db = smem_desc(v_addr + ks * 2048, 16384, 1024);
-          mma_ss(tm_o, da, db, idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
-        }
-        mma_commit(&bars[B_PVDONE]);
-        mma_commit(&bars[B_KVEMPTY + s]);
-      };
-      mbar_wait(&bars[B_QFULL], 0, abort_flag, a.status);
-      for (int j = 0; j < T; ++j) {
-        const int s = j % kStages, b = j & 1;
-        mbar_wait(&bars[B_KFULL + s], (j / kStages) & 1, abort_flag, a.status);
-        if (j >= 2) mbar_wait(&bars[B_SFREE + b], ((j >> 1) - 1) & 1, abort_flag, a.status);
-        tc_fence_after();
-        const uint32_t k_addr = smem_u32(sm + L::kK + s * L::kTileBytes);
+      auto kv_addr = [&](int e) { return smem_u32(sm + L::kKV + (e % kKvStages) * L::kTileBytes); };
+      auto wait_kv = [&](int e) { mbar_wait(&bars[B_KVFULL + e % kKvStages], (e / kKvStages) & 1, abort_flag, a.status); };
+      auto issue_qk = [&](int x, int j) {   // S_x = Q_x K_j^T
+        const uint32_t q_addr = smem_u32(sm + L::kQ + x * L::kTileBytes), k_addr = kv_addr(2 * j);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint64_t da = smem_desc(q_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
           const uint64_t db = smem_desc(k_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
-          mma_ss(tm_s[b], da, db, idesc_qk, ks > 0 ? 1u : 0u);
+          mma_ss(tm_s[x], da, db, idesc_qk, ks > 0 ? 1u : 0u);
         }
-        mma_commit(&bars[B_SFULL + b]);
-        if (j >= 1) issue_pv(j - 1);
+        mma_commit(&bars[B_SFULL + x]);
+      };
+      auto issue_pv = [&](int x, int j) {   // O_x += P_x V_j, P_x read from tensor memory (over S_x)
+        mbar_wait(&bars[B_PFULL + x], j & 1, abort_flag, a.status);
+        tc_fence_after();
+        const uint32_t v_addr = kv_addr(2 * j + 1);
+#pragma unroll
+        for (int ks = 0; ks < kTileN / 16; ++ks) {
+          const uint64_t db = smem_desc(v_addr + ks * 2048, 16384, 1024);
+          mma_ts(tm_o[x], tm_s[x] + ks * 8, db, idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+        }
+        mma_commit(&bars[B_ODONE + x]);
+      };
+      mbar_wait(&bars[B_QFULL + 0], 0, abort_flag, a.status);
+      if (active_b) mbar_wait(&bars[B_QFULL + 1], 0, abort_flag, a.status);
+      wait_kv(0);
+      tc_fence_after();
+      issue_qk(0, 0);
+      if (active_b) issue_qk(1, 0);
+      mma_commit(&bars[B_KVEMPTY + 0]);
+      for (int j = 1; j <= t_max; ++j) {       // products of key tile j-1, logits of key tile j
+        wait_kv(2 * j - 1);
+        if (j < t_max) wait_kv(2 * j);
+        tc_fence_after();
+        if (j - 1 < T[0]) issue_pv(0, j - 1);
+        if (j < T[0]) issue_qk(0, j);
+        if (active_b) {
+          issue_pv(1, j - 1);
+          if (j < T[1]) issue_qk(1, j);
+        }
+        mma_commit(&bars[B_KVEMPTY + (2 * j - 1) % kKvStages]);
+        if (j < t_max) mma_commit(&bars[B_KVEMPTY + (2 * j) % kKvStages]);
       }
-      issue_pv(T - 1);
     }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue: thread = query row
-    const int quad = warp & 3;
-    const int r = quad * 32 + lane;               // row inside the tile == TMEM lane
-    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const int row = row0 + r;
-    const int i_row = min(a.I - 1, i0 + r / a.g);  // rows past the block's end behave like its last input
-    float m_used = -INFINITY, l = 0.f;
-    unsigned char* sP = sm + L::kP;
-    for (int j = 0; j < T; ++j) {
-      const int b = j & 1;
-      mbar_wait(&bars[B_SFULL + b], (j >> 1) & 1, abort_flag, a.status);
-      tc_fence_after();
-      float sv[kTileN];
+    const int x = warp >> 2;                      // tile A or B
+    if (x == 0 || active_b) {
+      const int quad = warp & 3;
+      const int r = quad * 32 + lane;             // row inside the tile == TMEM lane
+      const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+      const int row = row0[x] + r;
+      const int i_row = min(a.I - 1, i0[x] + r / a.g);  // rows past the block's end behave like its last input
+      float m_used = -INFINITY, l = 0.f;
+      for (int j = 0; j < T[x]; ++j) {
+        mbar_wait(&bars[B_SFULL + x], j & 1, abort_flag, a.status);
+        tc_fence_after();
+        // visible columns of this key tile for this row
+        const int nvis = (j < t_old) ? min(kTileN, a.n_old - j * kTileN)
+                                     : max(0, min(kTileN, i_row - (j - t_old) * kTileN + 1));
+        float mx = -INFINITY;
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t raw[32];
-        tmem_ld32(tm_s[b] + lane_addr + cc * 32, raw);
-        tmem_wait_ld();
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t raw[32];
+          tmem_ld32(tm_s[x] + lane_addr + cc * 32, raw);
+          tmem_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 32; ++e) sv[cc * 32 + e] = __uint_as_float(raw[e]);
-      }
-      tc_fence_before();
-      mbar_arrive(&bars[B_SFREE + b]);
-      // number of visible columns of this tile for this row
-      const int nvis = (j < t_old) ? min(kTileN, a.n_old - j * kTileN)
-                                   : max(0, min(kTileN, i_row - (j - t_old) * kTileN + 1));
-      float mx = -INFINITY;
-#pragma unroll
-      for (int e = 0; e < kTileN; ++e) mx = fmaxf(mx, e < nvis ? sv[e] : -INFINITY);
-      const float mx2 = mx * a.scale_log2;
-      float alpha = 1.f;
-      bool rescale = false;
-      if (j == 0) m_used = mx2;
-      else if (mx2 > m_used + kRescaleThreshold) { alpha = ex2(m_used - mx2); m_used = mx2; rescale = true; }
-      if (j > 0) {
-        if (__any_sync(0xffffffffu, rescale)) {
-          // O is only safe to touch once the previous P V product has completed
-          mbar_wait(&bars[B_PVDONE], (j - 1) & 1, abort_flag, a.status);
-          tc_fence_after();
+          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, (cc * 32 + e < nvis) ? __uint_as_float(raw[e]) : -INFINITY);
+        }
+        const float mx2 = mx * a.scale_log2;
+        float alpha = 1.f;
+        bool rescale = false;
+        if (j == 0) m_used = mx2;
+        else if (mx2 > m_used + kRescaleThreshold) { alpha = ex2(m_used - mx2); m_used = mx2; rescale = true; }
+        // S_x(j) being complete implies the previous P.V into O_x has completed, so O_x may be touched here
+        if (j > 0 && __any_sync(0xffffffffu, rescale)) {
 #pragma unroll
           for (int cc = 0; cc < D / 32; ++cc) {
             uint32_t raw[32];
-            tmem_ld32(tm_o + lane_addr + cc * 32, raw);
+            tmem_ld32(tm_o[x] + lane_addr + cc * 32, raw);
             tmem_wait_ld();
 #pragma unroll
             for (int e = 0; e < 32; ++e) raw[e] = __float_as_uint(__uint_as_float(raw[e]) * alpha);
-            tmem_st32(tm_o + lane_addr + cc * 32, raw);
+            tmem_st32(tm_o[x] + lane_addr + cc * 32, raw);
           }
-          tmem_wait_st();
           l *= alpha;
         }
-      }
-      float psum = 0.f;
+        float psum = 0.f;
 #pragma unroll
-      for (int e = 0; e < kTileN; ++e) {
-        const float p = e < nvis ? ex2(fmaf(sv[e], a.scale_log2, -m_used)) : 0.f;
-        sv[e] = p;
-        psum += p;
-      }
-      l += psum;
-      if (j > 0) mbar_wait(&bars[B_PVDONE], (j - 1) & 1, abort_flag, a.status);  // previous product done with sP
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t raw[32];
+          tmem_ld32(tm_s[x] + lane_addr + cc * 32, raw);
+          tmem_wait_ld();
+          uint32_t pk[16];
 #pragma unroll
-      for (int pc = 0; pc < kTileN / 8; ++pc) {
-        uint4 w;
-        w.x = pack_bf16(sv[pc * 8 + 0], sv[pc * 8 + 1]);
-        w.y = pack_bf16(sv[pc * 8 + 2], sv[pc * 8 + 3]);
-        w.z = pack_bf16(sv[pc * 8 + 4], sv[pc * 8 + 5]);
-        w.w = pack_bf16(sv[pc * 8 + 6], sv[pc * 8 + 7]);
-        *reinterpret_cast<uint4*>(sP + (pc >> 3) * 16384 + sw128_offset(r, pc & 7)) = w;
+          for (int e = 0; e < 16; ++e) {
+            const int c0 = cc * 32 + 2 * e;
+            const float p0 = (c0 < nvis) ? ex2(fmaf(__uint_as_float(raw[2 * e]), a.scale_log2, -m_used)) : 0.f;
+            const float p1 = (c0 + 1 < nvis) ? ex2(fmaf(__uint_as_float(raw[2 * e + 1]), a.scale_log2, -m_used)) : 0.f;
+            psum += p0 + p1;
+            pk[e] = pack_bf16(p0, p1);
+          }
+          // bf16 pairs of columns [32cc, 32cc+32) land in columns [16cc, 16cc+16): logits already consumed
+          tmem_st16(tm_s[x] + lane_addr + cc * 16, pk);
+        }
+        l += psum;
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bars[B_PFULL + x]);
       }
-      fence_async_smem();
-      tc_fence_before();
-      mbar_arrive(&bars[B_PFULL]);
-    }
-    // epilogue: O / l -> bf16, log2-sum-exp
-    mbar_wait(&bars[B_PVDONE], (T - 1) & 1, abort_flag, a.status);
-    tc_fence_after();
-    const float inv = 1.f / l;
-    const bool live = row < R;
-    const int ii = row / a.g, hh = row % a.g;
-    __nv_bfloat16* op = reinterpret_cast<__nv_bfloat16*>(a.out) + ((size_t)(smp * a.I + ii) * a.Hq + kh * a.g + hh) * D;
+      // epilogue: O / l -> bf16 -> swizzled tile in the (now idle) query buffer -> TMA store; log2-sum-exp
+      mbar_wait(&bars[B_ODONE + x], (T[x] - 1) & 1, abort_flag, a.status);
+      tc_fence_after();
+      const float inv = 1.f / l;
+      unsigned char* stage = sm + L::kQ + x * L::kTileBytes;
 #pragma unroll
-    for (int cc = 0; cc < D / 32; ++cc) {
-      uint32_t raw[32];
-      tmem_ld32(tm_o + lane_addr + cc * 32, raw);
-      tmem_wait_ld();
-      if (live) {
+      for (int cc = 0; cc < D / 32; ++cc) {
+        uint32_t raw[32];
+        tmem_ld32(tm_o[x] + lane_addr + cc * 32, raw);
+        tmem_wait_ld();
 #pragma unroll
         for (int q4 = 0; q4 < 4; ++q4) {
           uint4 w;
@@ -255,21 +263,29 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
           w.y = pack_bf16(__uint_as_float(raw[q4 * 8 + 2]) * inv, __uint_as_float(raw[q4 * 8 + 3]) * inv);
           w.z = pack_bf16(__uint_as_float(raw[q4 * 8 + 4]) * inv, __uint_as_float(raw[q4 * 8 + 5]) * inv);
           w.w = pack_bf16(__uint_as_float(raw[q4 * 8 + 6]) * inv, __uint_as_float(raw[q4 * 8 + 7]) * inv);
-          *reinterpret_cast<uint4*>(op + cc * 32 + q4 * 8) = w;
+          const int piece = cc * 4 + q4;            // 16-byte piece of the row: chunk = piece / 8
+          *reinterpret_cast<uint4*>(stage + (piece >> 3) * 16384 + sw128_offset(r, piece & 7)) = w;
         }
       }
+      if (row < R) a.lse2[(size_t)unit * R + row] = m_used + log2f(l);
+      fence_async_smem();
+      named_bar_sync(1 + x, 128);
+      if (r == 0) {
+        for (int c = 0; c < L::kChunks; ++c) tma_store_5d(&maps.o, stage + c * 16384, c * 64, 0, kh, i0[x], smp);
+        tma_store_commit_and_wait();
+      }
     }
-    if (live) a.lse2[(size_t)unit * R + row] = m_used + log2f(l);
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+  if (warp == 8) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ------------------------------------------------------------------------------------------------------
 // Score pass.  CTA = (tile of 128 candidate keys, unit).  A = the key tile (loaded once), B = the unit's query
-// tiles streamed through a ring; S^T lands in TMEM with lane = key, column = query row.
-constexpr int kScoreThreads = 192;
+// tiles streamed through a ring; S^T lands in TMEM with lane = key, column = query row.  Two reducer
+// warpgroups take alternate query tiles (one TMEM buffer each); their partial sums are added in a fixed order.
+constexpr int kScoreThreads = 320;   // warps 0-3, 4-7: reducers; warp 8: MMA + TMEM owner; warp 9: TMA
 constexpr int kQStages = 3;
 
 template <int D>
@@ -279,7 +295,8 @@ struct ScoreSmem {
   static constexpr int kK = 0;
   static constexpr int kQ = kK + kTileBytes;
   static constexpr int kLse = kQ + kQStages * kTileBytes;      // 2 x 128 floats
-  static constexpr int kBars = kLse + 2 * 128 * 4;
+  static constexpr int kPart = kLse + 2 * 128 * 4;             // 128 floats: warpgroup 1's partial sums
+  static constexpr int kBars = kPart + 128 * 4;
   static constexpr int kTotal = kBars + 256 + 1024;
 };
 enum { C_KFULL = 0, C_QFULL = 1, C_QEMPTY = C_QFULL + kQStages, C_SFULL = C_QEMPTY + kQStages, C_SFREE = C_SFULL + 2,
@@ -295,6 +312,7 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + C_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float* sLse = reinterpret_cast<float*>(sm + L::kLse);
+  float* sPart = reinterpret_cast<float*>(sm + L::kPart);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int unit = blockIdx.y, smp = unit / a.Hkv, kh = unit % a.Hkv;
@@ -315,14 +333,14 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
     for (int b = 0; b < 2; ++b) { mbar_init(&bars[C_SFULL + b], 1); mbar_init(&bars[C_SFREE + b], 128); }
     mbar_fence_init();
   }
-  if (warp == 1) tmem_alloc(tmem_slot, 256);
+  if (warp == 8) tmem_alloc(tmem_slot, 256);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tm_s[2] = {tmem, tmem + 128};
 
-  if (warp == 0) {
+  if (warp == 9) {
     if (lane == 0) {
       mbar_expect_tx(&bars[C_KFULL], L::kTileBytes);
       for (int c = 0; c < L::kChunks; ++c) {
@@ -338,7 +356,7 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
                       &bars[C_QFULL + s]);
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == 8) {
     if (lane == 0) {
       const uint32_t idesc = instr_desc(kTileN, kTileM, 0, 0);
       const uint32_t k_addr = smem_u32(sm + L::kK);
@@ -360,48 +378,60 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
       }
     }
   } else {
+    const int wg = warp >> 2;                      // reducer warpgroup: takes query tiles t = wg, wg + 2, ...
     const int quad = warp & 3;
     const int key = quad * 32 + lane;              // key inside the tile == TMEM lane
     const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
-    const int t128 = tid - 64;                     // 0..127 among the reducer threads
     float acc = 0.f;
-    for (int t = 0; t < T; ++t) {
-      const int b = t & 1;
+    for (int t = wg; t < T; t += 2) {
       const int qrow0 = (qt0 + t) * kTileM;
       // this tile's log2-sum-exp values; +inf for rows past the block's end (weight 0)
       {
-        const int rr = qrow0 + t128;
-        sLse[b * 128 + t128] = rr < R ? a.lse2[(size_t)unit * R + rr] : INFINITY;
+        const int rr = qrow0 + key;
+        sLse[wg * 128 + key] = rr < R ? a.lse2[(size_t)unit * R + rr] : INFINITY;
       }
-      named_bar_sync(1, 128);
-      mbar_wait(&bars[C_SFULL + b], (t >> 1) & 1, abort_flag, a.status);
+      named_bar_sync(1 + wg, 128);
+      mbar_wait(&bars[C_SFULL + wg], (t >> 1) & 1, abort_flag, a.status);
       tc_fence_after();
       // first query row of the tile that may see this key (causal mask inside the block)
       const int first_vis = is_old ? 0 : max(0, (c0 + key) * a.g - qrow0);
       float part = 0.f;
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        uint32_t raw[32];
-        tmem_ld32(tm_s[b] + lane_addr + cc * 32, raw);
+      for (int half = 0; half < 2; ++half) {
+        uint32_t ra[32], rb[32];
+        tmem_ld32(tm_s[wg] + lane_addr + half * 64, ra);
+        tmem_ld32(tm_s[wg] + lane_addr + half * 64 + 32, rb);
         tmem_wait_ld();
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
-          const int col = cc * 32 + e;
-          const float p = ex2(fmaf(__uint_as_float(raw[e]), a.scale_log2, -sLse[b * 128 + col]));
+          const int col = half * 64 + e;
+          const float p = ex2(fmaf(__uint_as_float(ra[e]), a.scale_log2, -sLse[wg * 128 + col]));
+          part += col >= first_vis ? p : 0.f;
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const int col = half * 64 + 32 + e;
+          const float p = ex2(fmaf(__uint_as_float(rb[e]), a.scale_log2, -sLse[wg * 128 + col]));
           part += col >= first_vis ? p : 0.f;
         }
       }
       acc += part;
       tc_fence_before();
-      mbar_arrive(&bars[C_SFREE + b]);
+      mbar_arrive(&bars[C_SFREE + wg]);
+      named_bar_sync(1 + wg, 128);                 // everyone is done with this tile's sLse before it is rewritten
     }
-    const int j = is_old ? kt * kTileN + key : c0 + key;
-    if (is_old) { if (j < a.n_old) a.sum_weights[(size_t)unit * a.cap + j] += acc; }
-    else if (j < a.I) a.new_sum[(size_t)unit * a.I + j] = acc;
+    if (wg == 1) sPart[key] = acc;
+    named_bar_sync(3, 256);
+    if (wg == 0) {
+      acc += sPart[key];
+      const int j = is_old ? kt * kTileN + key : c0 + key;
+      if (is_old) { if (j < a.n_old) a.sum_weights[(size_t)unit * a.cap + j] += acc; }
+      else if (j < a.I) a.new_sum[(size_t)unit * a.I + j] = acc;
+    }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, 256);
+  if (warp == 8) tmem_dealloc(tmem, 256);
 }
 
 // ------------------------------------------------------------------------------------------------------
@@ -431,7 +461,8 @@ bool encode(CUtensorMap* m, const void* base, int rank, const cuuint64_t* dims, 
                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tensor maps of one call.  Rows past n_old (slab) or past I (block, queries) read as zeros.
+// Tensor maps of one call.  Rows past n_old (slab) or past I (block, queries) read as zeros; output rows past I
+// are clipped.
 bool build_maps(int d, const CacheView& c, const BlockArgs& a, TcMaps* m) {
   const cuuint64_t D = (cuuint64_t)d, e = 2;
   const cuuint64_t units = (cuuint64_t)c.nsamples * c.Hkv;
@@ -440,6 +471,7 @@ bool build_maps(int d, const CacheView& c, const BlockArgs& a, TcMaps* m) {
     cuuint64_t str[4] = {D * e, (cuuint64_t)c.g * D * e, (cuuint64_t)c.Hq * D * e, (cuuint64_t)a.I * c.Hq * D * e};
     cuuint32_t box[5] = {64, (cuuint32_t)c.g, 1, (cuuint32_t)(kTileM / c.g), 1};
     if (!encode(&m->q, a.q, 5, dims, str, box)) return false;
+    if (!encode(&m->o, a.out, 5, dims, str, box)) return false;
   }
   {
     cuuint64_t dims[3] = {D, (cuuint64_t)(c.n_old > 0 ? c.n_old : 1), units};
@@ -462,7 +494,7 @@ TcArgs make_args(const CacheView& c, const BlockArgs& a) {
   TcArgs t;
   t.n_old = c.n_old; t.I = a.I; t.g = c.g; t.Hq = c.Hq; t.Hkv = c.Hkv;
   t.scale_log2 = a.scale * kLog2e;
-  t.out = a.out; t.lse2 = a.lse; t.sum_weights = c.sum_weights; t.new_sum = a.new_sum;
+  t.lse2 = a.lse; t.sum_weights = c.sum_weights; t.new_sum = a.new_sum;
   t.cap = c.cap; t.status = c.status;
   return t;
 }
@@ -480,7 +512,7 @@ cudaError_t launch_fwd_t(const CacheView& c, const BlockArgs& a, cudaStream_t st
     configured = true;
   }
   const int R = a.I * c.g;
-  dim3 grid((R + kTileM - 1) / kTileM, c.nsamples * c.Hkv);
+  dim3 grid((R + 2 * kTileM - 1) / (2 * kTileM), c.nsamples * c.Hkv);
   ProfileScope prof(kAttnFwd, st);
   attn_fwd_tc<D><<<grid, kFwdThreads, FwdSmem<D>::kTotal, st>>>(g_maps, make_args(c, a));
   count_launch();
