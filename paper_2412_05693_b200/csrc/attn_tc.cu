@@ -196,14 +196,27 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
         // visible columns of this key tile for this row
         const int nvis = (j < t_old) ? min(kTileN, a.n_old - j * kTileN)
                                      : max(0, min(kTileN, i_row - (j - t_old) * kTileN + 1));
+        const bool full = __all_sync(0xffffffffu, nvis >= kTileN);   // warp-uniform: nothing to mask in this tile
         float mx = -INFINITY;
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          uint32_t raw[32];
-          tmem_ld32(tm_s[x] + lane_addr + cc * 32, raw);
+        for (int hh = 0; hh < 2; ++hh) {                              // two TMEM loads in flight
+          uint32_t ra[32], rb[32];
+          tmem_ld32(tm_s[x] + lane_addr + hh * 64, ra);
+          tmem_ld32(tm_s[x] + lane_addr + hh * 64 + 32, rb);
           tmem_wait_ld();
+          if (full) {
 #pragma unroll
-          for (int e = 0; e < 32; ++e) mx = fmaxf(mx, (cc * 32 + e < nvis) ? __uint_as_float(raw[e]) : -INFINITY);
+            for (int e = 0; e < 32; e += 2) {
+              mx = max3(mx, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+              mx = max3(mx, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              mx = fmaxf(mx, (hh * 64 + e < nvis) ? __uint_as_float(ra[e]) : -INFINITY);
+              mx = fmaxf(mx, (hh * 64 + 32 + e < nvis) ? __uint_as_float(rb[e]) : -INFINITY);
+            }
+          }
         }
         const float mx2 = mx * a.scale_log2;
         float alpha = 1.f;
@@ -223,25 +236,38 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
           }
           l *= alpha;
         }
-        float psum = 0.f;
+        float ps0 = 0.f, ps1 = 0.f;
+        const float neg_m = -m_used;
+        uint32_t cur[32], nxt[32];
+        tmem_ld32(tm_s[x] + lane_addr, cur);
+        tmem_wait_ld();
 #pragma unroll
         for (int cc = 0; cc < 4; ++cc) {
-          uint32_t raw[32];
-          tmem_ld32(tm_s[x] + lane_addr + cc * 32, raw);
-          tmem_wait_ld();
+          if (cc < 3) tmem_ld32(tm_s[x] + lane_addr + (cc + 1) * 32, nxt);   // next chunk loads while this one is used
           uint32_t pk[16];
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const int c0 = cc * 32 + 2 * e;
-            const float p0 = (c0 < nvis) ? ex2(fmaf(__uint_as_float(raw[2 * e]), a.scale_log2, -m_used)) : 0.f;
-            const float p1 = (c0 + 1 < nvis) ? ex2(fmaf(__uint_as_float(raw[2 * e + 1]), a.scale_log2, -m_used)) : 0.f;
-            psum += p0 + p1;
+            float x0, x1;
+            fma2(x0, x1, __uint_as_float(cur[2 * e]), __uint_as_float(cur[2 * e + 1]), a.scale_log2, neg_m);
+            float p0 = ex2(x0), p1 = ex2(x1);
+            if (!full) {
+              const int c0 = cc * 32 + 2 * e;
+              p0 = (c0 < nvis) ? p0 : 0.f;
+              p1 = (c0 + 1 < nvis) ? p1 : 0.f;
+            }
+            ps0 += p0;
+            ps1 += p1;
             pk[e] = pack_bf16(p0, p1);
           }
           // bf16 pairs of columns [32cc, 32cc+32) land in columns [16cc, 16cc+16): logits already consumed
           tmem_st16(tm_s[x] + lane_addr + cc * 16, pk);
+          if (cc < 3) {
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) cur[e] = nxt[e];
+          }
         }
-        l += psum;
+        l += ps0 + ps1;
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&bars[B_PFULL + x]);
