@@ -28,7 +28,7 @@ METRIC = "P&D evicting-attention tokens/s at max batch; % of TC (prefill) / HBM 
 UNIT = "tokens/s"
 # DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
 # capture, see profiles/); None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"attn_fwd": None}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": 91.9e6}   # steady-state launch, profiles/attn_fwd_tc_cfg2_traffic.md
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -318,7 +318,7 @@ def main():
         flops_per_step = 4.0 * wl.d * prefill_pairs(wl) * wl.b * wl.Hq * wl.L
         achieved = flops_per_step / (attn_ms * 1e-3) / 1e12 if attn_ms > 0 else 0.0
         peak = pk["bf16_tflops_sustained"] if wl.dtype == "bf16" else pk["bf16_tflops_sustained"] / 2
-        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get("attn_fwd")
+        traffic = NCU_TRAFFIC_BYTES_PER_LAUNCH.get(wl.name)
         roofline = {"bound": "tensor", "kernel": "prefill-block attention forward", "achieved": achieved,
                     "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic,
                     "peak_source": f"{pk_src} (sustained bf16 matmul)", "launches_per_step": attn_n,
