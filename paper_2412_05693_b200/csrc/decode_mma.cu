@@ -123,72 +123,117 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
   const int n_iter = (n1 + kRowsPerIter - 1) / kRowsPerIter;   // same trip count for every thread
 
   // ---- logits (log2 domain).  Tile rows gid and gid+8; the k-slots of thread tq are its own 8 elements.
-  for (int it = 0; it < n_iter; ++it) {
-    const int tb = it * kRowsPerIter + warp * 16;
-    const int j0 = tb + gid, j1 = tb + gid + 8;
+  // The loads of iteration it+1 are issued before the MMAs of iteration it (one round trip in flight).
+  auto load_k = [&](int it, uint4 (&xx)[QR], uint4 (&yy)[QR]) {
+    const int j0 = it * kRowsPerIter + warp * 16 + gid, j1 = j0 + 8;
+#pragma unroll
+    for (int r = 0; r < QR; ++r) {
+      xx[r] = ldg16_or_zero(kslab + (size_t)j0 * D + 32 * r + 8 * tq, j0 < n1);
+      yy[r] = ldg16_or_zero(kslab + (size_t)j1 * D + 32 * r + 8 * tq, j1 < n1);
+    }
+  };
+  // rows of V for iteration `it`: thread (gid, tq) loads, from the 4 rows tb + 4tq + {0..3}, elements [64r + 8gid, +8)
+  auto load_v = [&](int it, uint4 (&zz)[VR][4]) {
+    const int jr = it * kRowsPerIter + warp * 16 + 4 * tq;
+#pragma unroll
+    for (int r = 0; r < VR; ++r)
+#pragma unroll
+      for (int sx = 0; sx < 4; ++sx)
+        zz[r][sx] = ldg16_or_zero(vslab + (size_t)(jr + sx) * D + 64 * r + 8 * gid, jr + sx < n1);
+  };
+  {
     uint4 x[QR], y[QR];
+    load_k(0, x, y);
+    for (int it = 0; it < n_iter; ++it) {
+      const int j0 = it * kRowsPerIter + warp * 16 + gid, j1 = j0 + 8;
+      uint4 xn[QR], yn[QR];
+      if (it + 1 < n_iter) load_k(it + 1, xn, yn);
+      float cacc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int r = 0; r < QR; ++r) {
-      x[r] = ldg16_or_zero(kslab + (size_t)j0 * D + 32 * r + 8 * tq, j0 < n1);
-      y[r] = ldg16_or_zero(kslab + (size_t)j1 * D + 32 * r + 8 * tq, j1 < n1);
-    }
-    float cacc[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int r = 0; r < QR; ++r) {
+        mma16816(cacc, x[r].x, y[r].x, x[r].y, y[r].y, qf[r][0], qf[r][1]);
+        mma16816(cacc, x[r].z, y[r].z, x[r].w, y[r].w, qf[r][2], qf[r][3]);
+      }
+      // cacc[0], cacc[1]: key j0, heads 2tq, 2tq+1 ; cacc[2], cacc[3]: key j1
+      if (2 * tq < G) {
+        if (j0 < n1) s.p[(2 * tq) * n1t + j0] = cacc[0] * sc2;
+        if (j1 < n1) s.p[(2 * tq) * n1t + j1] = cacc[2] * sc2;
+      }
+      if (2 * tq + 1 < G) {
+        if (j0 < n1) s.p[(2 * tq + 1) * n1t + j0] = cacc[1] * sc2;
+        if (j1 < n1) s.p[(2 * tq + 1) * n1t + j1] = cacc[3] * sc2;
+      }
+      if (it + 1 < n_iter) {
 #pragma unroll
-    for (int r = 0; r < QR; ++r) {
-      mma16816(cacc, x[r].x, y[r].x, x[r].y, y[r].y, qf[r][0], qf[r][1]);
-      mma16816(cacc, x[r].z, y[r].z, x[r].w, y[r].w, qf[r][2], qf[r][3]);
+        for (int r = 0; r < QR; ++r) { x[r] = xn[r]; y[r] = yn[r]; }
+      }
     }
-    // cacc[0], cacc[1]: key j0, heads 2tq, 2tq+1 ; cacc[2], cacc[3]: key j1
-    if (2 * tq < G) {
-      if (j0 < n1) s.p[(2 * tq) * n1t + j0] = cacc[0] * sc2;
-      if (j1 < n1) s.p[(2 * tq) * n1t + j1] = cacc[2] * sc2;
-    }
-    if (2 * tq + 1 < G) {
-      if (j0 < n1) s.p[(2 * tq + 1) * n1t + j0] = cacc[1] * sc2;
-      if (j1 < n1) s.p[(2 * tq + 1) * n1t + j1] = cacc[3] * sc2;
-    }
+  }
+  // first V tile and the old sum_weights start loading now; they are needed only after the softmax
+  uint4 z[VR][4];
+  load_v(0, z);
+  constexpr int kSwPrefetch = 4;
+  float sw_old[kSwPrefetch];
+#pragma unroll
+  for (int u = 0; u < kSwPrefetch; ++u) {
+    const int j = tid + u * kThreads;
+    sw_old[u] = (j < c.n_old) ? c.sum_weights[base + j] : 0.f;
   }
   __syncthreads();
 
-  // ---- softmax over the n1 rows, per head
+  // ---- softmax over the n1 rows; the G heads are reduced side by side (independent shuffle chains)
   float inv[G];
+  {
+    float m[G], t[G];
 #pragma unroll
-  for (int h = 0; h < G; ++h) {
-    float m = -INFINITY;
-    for (int j = tid; j < n1; j += kThreads) m = fmaxf(m, s.p[h * n1t + j]);
+    for (int h = 0; h < G; ++h) m[h] = -INFINITY;
+    for (int j = tid; j < n1; j += kThreads)
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-    if (lane == 0) s.wred[h * kWarps + warp] = m;
-  }
-  __syncthreads();
+      for (int h = 0; h < G; ++h) m[h] = fmaxf(m[h], s.p[h * n1t + j]);
 #pragma unroll
-  for (int h = 0; h < G; ++h) {
-    float m = -INFINITY;
+    for (int off = 16; off > 0; off >>= 1)
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) m = fmaxf(m, s.wred[h * kWarps + w]);
-    float t = 0.f;
-    for (int j = tid; j < n1; j += kThreads) {
-      const float e = ex2f(s.p[h * n1t + j] - m);
-      s.p[h * n1t + j] = e;
-      t += e;
+      for (int h = 0; h < G; ++h) m[h] = fmaxf(m[h], __shfl_xor_sync(0xffffffffu, m[h], off));
+    if (lane == 0)
+#pragma unroll
+      for (int h = 0; h < G; ++h) s.wred[h * kWarps + warp] = m[h];
+    __syncthreads();
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      float mm = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) mm = fmaxf(mm, s.wred[h * kWarps + w]);
+      m[h] = mm;
+      t[h] = 0.f;
     }
+    for (int j = tid; j < n1; j += kThreads)
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
-    if (lane == 0) s.wred[(G + h) * kWarps + warp] = t;
-  }
-  __syncthreads();
+      for (int h = 0; h < G; ++h) {
+        const float e = ex2f(s.p[h * n1t + j] - m[h]);
+        s.p[h * n1t + j] = e;
+        t[h] += e;
+      }
 #pragma unroll
-  for (int h = 0; h < G; ++h) {
-    float t = 0.f;
+    for (int off = 16; off > 0; off >>= 1)
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) t += s.wred[(G + h) * kWarps + w];  // fixed order
-    inv[h] = 1.f / t;
+      for (int h = 0; h < G; ++h) t[h] += __shfl_xor_sync(0xffffffffu, t[h], off);
+    if (lane == 0)
+#pragma unroll
+      for (int h = 0; h < G; ++h) s.wred[(G + h) * kWarps + warp] = t[h];
+    __syncthreads();
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+      float tt = 0.f;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) tt += s.wred[(G + h) * kWarps + w];  // fixed order
+      inv[h] = 1.f / tt;
+    }
   }
 
   // ---- normalise, sum_weights += attn_weights (heads added in a fixed order), candidate for eviction
   float best_ave = INFINITY;
   int best_j = -1;
-  for (int j = tid; j < n1t; j += kThreads) {
+  for (int j = tid, u = 0; j < n1t; j += kThreads, ++u) {
     if (j >= n1) {
 #pragma unroll
       for (int h = 0; h < G; ++h) s.p[h * n1t + j] = 0.f;   // padding keys carry no weight
@@ -201,7 +246,14 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
       s.p[h * n1t + j] = p;
       add += p;
     }
-    const float sw = ((j < c.n_old) ? c.sum_weights[base + j] : 0.f) + add;
+    float old_sw = 0.f;
+    if (u < kSwPrefetch) {
+#pragma unroll
+      for (int uu = 0; uu < kSwPrefetch; ++uu) old_sw = (uu == u) ? sw_old[uu] : old_sw;
+    } else if (j < c.n_old) {
+      old_sw = c.sum_weights[base + j];
+    }
+    const float sw = old_sw + add;
     s.score[j] = sw;
     if (evict_one) {
       const float ave = sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
@@ -251,12 +303,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
   for (int it = 0; it < n_iter; ++it) {
     const int tb = it * kRowsPerIter + warp * 16;
     const int jr = tb + 4 * tq;   // first of this thread's 4 rows
-    uint4 z[VR][4];
-#pragma unroll
-    for (int r = 0; r < VR; ++r)
-#pragma unroll
-      for (int sx = 0; sx < 4; ++sx)
-        z[r][sx] = ldg16_or_zero(vslab + (size_t)(jr + sx) * D + 64 * r + 8 * gid, jr + sx < n1);
+    uint4 zn[VR][4];
+    if (it + 1 < n_iter) load_v(it + 1, zn);   // next iteration's rows load while this one is multiplied
     // p^T fragment: (head gid; keys jr, jr+1) and (head gid; keys jr+2, jr+3)
     uint32_t pb0 = 0u, pb1 = 0u;
     if (gid < G && jr < n1t) {
@@ -286,6 +334,12 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
           const int j = jr + sx;
           if (j < n1 && j > hole) st_global_16(vslab + (size_t)(j - 1) * D + 64 * r + 8 * gid, z[r][sx]);
         }
+    }
+    if (it + 1 < n_iter) {
+#pragma unroll
+      for (int r = 0; r < VR; ++r)
+#pragma unroll
+        for (int sx = 0; sx < 4; ++sx) z[r][sx] = zn[r][sx];
     }
   }
   // K rows behind the hole: one-row shift (re-read, mostly from L2: the logits pass just streamed them)
