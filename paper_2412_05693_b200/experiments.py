@@ -1,0 +1,185 @@
+"""Whole-workload runs at the paper-scale batch sizes (one JSON line per run on stdout).
+
+    python -m paper_2412_05693_b200.experiments --run cfg3_max      # P&D arm at the batch that fills 40 GiB
+    python -m paper_2412_05693_b200.experiments --run cfg3_ratio    # P&D vs decode-only compression, same arena
+    python -m paper_2412_05693_b200.experiments --run cfg4          # 32 layers, batch that fills 120 GiB
+    python -m paper_2412_05693_b200.experiments --run cfg5          # the six (block, kv_max) combinations
+
+Batches this large cannot keep their prompts resident (one block of cfg3 at b = 10072 is 63 GB of Q/K/V), so
+inputs are drawn on the fly per (layer, block, range of samples) from the seeded generator and every library
+call is timed on its own with CUDA events; generation time is outside the timed regions.  Only the C-ABI
+library runs inside them.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2412_05693_b200 import BatchMaxCache, Config, arena_bytes, max_batch  # noqa: E402
+from paper_2412_05693_b200.workloads import CFG5_SWEEP, WORKLOADS, Inputs, Workload  # noqa: E402
+
+GiB = 2 ** 30
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), float(d["bf16_tflops_sustained"]), "measured"
+    return 6650.0, 1400.0, "fallback"
+
+
+def make_cfg(wl: Workload, batch: int, arm: str, micro: int, device: int = 0) -> Config:
+    growth = max(1, wl.p_dec) if arm == "pd" else wl.s + max(1, wl.p_dec) - wl.K
+    return Config(batch=batch, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.d, kv_max=wl.K, block_max=wl.B,
+                  growth=growth, dtype=wl.dtype, n_layers=wl.L, device=device, max_call_samples=micro)
+
+
+class Timer:
+    def __init__(self):
+        self.pairs = []
+
+    def __call__(self, fn):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        self.pairs.append((e0, e1))
+
+    def total_ms(self):
+        torch.cuda.synchronize()
+        t = sum(a.elapsed_time(b) for a, b in self.pairs)
+        self.pairs = []
+        return t
+
+
+def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=None, device: int = 0):
+    """One arm over the whole schedule.  arm 'pd': evict to K after every block and decode step (P&D);
+    arm 'do': cache the whole prompt, compress to K once after it, then decode with eviction (decode-only
+    compression, Sec. 1).  Returns a dict of timings and derived rates."""
+    wl = wl.with_(b=batch)
+    cfg = make_cfg(wl, batch, arm, micro, device)
+    dev = torch.device("cuda", device)
+    need = arena_bytes(cfg)
+    if arena is None:
+        arena = torch.empty(need, dtype=torch.uint8, device=dev)
+    assert arena.numel() >= need, "arena smaller than the memory model asks for"
+    cache = BatchMaxCache(cfg, arena=arena[:need])
+    inp = Inputs(wl, dev)
+    t_pre, t_dec = Timer(), Timer()
+    ms_pre = ms_dec = 0.0
+    layers = range(wl.L) if layers is None else layers
+    out_blk = torch.empty(micro, wl.B, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
+    out_dec = torch.empty(micro, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
+    pairs = 0
+    for layer in layers:
+        n = 0
+        for pos0 in range(0, wl.s, wl.B):
+            I = min(wl.B, wl.s - pos0)
+            ev = wl.K if arm == "pd" else -1
+            for s0 in range(0, batch, micro):
+                ns = min(micro, batch - s0)
+                q, k, v = inp.block(layer, pos0, I, s0, ns)
+                t_pre(lambda: cache.prefill_block(q, k, v, pos0, out=out_blk[:ns, :I], evict_to=ev, layer=layer,
+                                                  sample0=s0))
+            pairs += I * n + I * (I + 1) // 2
+            n = min(n + I, wl.K) if arm == "pd" else n + I
+            ms_pre += t_pre.total_ms()
+        if arm == "do":
+            for s0 in range(0, batch, micro):
+                ns = min(micro, batch - s0)
+                t_pre(lambda: cache.evict(wl.K, layer=layer, sample0=s0, nsamples=ns))
+            n = min(n, wl.K)
+            ms_pre += t_pre.total_ms()
+        for t in range(wl.steps):
+            full = n + 1 >= wl.K + wl.p_dec
+            ev = wl.K if full else -1
+            for s0 in range(0, batch, micro):
+                ns = min(micro, batch - s0)
+                q, k, v = inp.block(layer, wl.s + t, 1, s0, ns)
+                q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
+                t_dec(lambda: cache.decode_step(q, k, v, out=out_dec[:ns], evict_to=ev, layer=layer, sample0=s0))
+            n = wl.K if full else n + 1
+            if (t & 15) == 15 or t == wl.steps - 1:
+                ms_dec += t_dec.total_ms()
+    assert cache.status() == 0
+    n_layers = len(list(layers))
+    n_end, cur = cache.length(layer=list(layers)[-1], sample=batch - 1)
+    cache.close()
+    hbm, tf, src = peaks()
+    e = wl.elem_bytes
+    flops = 4.0 * wl.d * (pairs / n_layers) * batch * wl.Hq * n_layers
+    n1 = min(wl.K, wl.s) + 1
+    dec_bytes = batch * wl.Hkv * n_layers * wl.steps * (n1 * (2 * wl.d * e + 16) + 2 * wl.d * e + 2 * wl.g * wl.d * e)
+    res = {
+        "workload": wl.name, "arm": arm, "batch": batch, "layers_run": n_layers, "micro_batch": micro,
+        "arena_GiB": need / GiB, "final_n": n_end, "final_curr_id": cur,
+        "prefill_ms": ms_pre, "decode_ms": ms_dec,
+        "prefill_tok_s": batch * wl.s * n_layers / (ms_pre * 1e-3),
+        "decode_tok_s": batch * wl.steps * n_layers / (ms_dec * 1e-3) if ms_dec > 0 else None,
+        "generated_tok_s": batch * wl.steps * n_layers / ((ms_pre + ms_dec) * 1e-3),
+        "prefill_useful_tflops": flops / (ms_pre * 1e-3) / 1e12,
+        "prefill_frac_of_peak": flops / (ms_pre * 1e-3) / 1e12 / tf,
+        "decode_gbs": dec_bytes / (ms_dec * 1e-3) / 1e9 if ms_dec > 0 else None,
+        "decode_frac_of_peak": dec_bytes / (ms_dec * 1e-3) / 1e9 / hbm if ms_dec > 0 else None,
+        "peaks": {"hbm_gbs": hbm, "bf16_tflops_sustained": tf, "source": src},
+        "note": "prefill = all bm_prefill_block calls incl. score pass and eviction (whole call, not the forward kernel "
+                "alone); decode bytes exclude compaction moves; every call timed with its own CUDA events",
+    }
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--run", required=True, choices=["cfg3_max", "cfg3_ratio", "cfg4", "cfg5"])
+    ap.add_argument("--budget-gib", type=float, default=None)
+    ap.add_argument("--micro", type=int, default=256)
+    ap.add_argument("--layers", type=int, default=None, help="run only the first N layers (cfg4)")
+    ap.add_argument("--decode-steps", type=int, default=None)
+    args = ap.parse_args()
+    assert torch.cuda.is_available(), "needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(0)
+    if args.run in ("cfg3_max", "cfg3_ratio"):
+        wl = WORKLOADS["cfg3"]
+        if args.decode_steps is not None:
+            wl = wl.with_(steps=args.decode_steps)
+        budget = int((args.budget_gib or 40.0) * GiB)
+        b_pd = max_batch(make_cfg(wl, 1, "pd", args.micro), budget)
+        b_do = max_batch(make_cfg(wl, 1, "do", args.micro), budget)
+        arena = torch.empty(budget, dtype=torch.uint8, device="cuda")
+        res_pd = run_arm(wl, b_pd, "pd", args.micro, arena=arena)
+        out = {"run": args.run, "budget_GiB": budget / GiB, "b_pd": b_pd, "b_do": b_do,
+               "batch_ratio": b_pd / b_do, "predicted_ratio": (wl.s + 1) / (wl.K + 1), "pd": res_pd}
+        if args.run == "cfg3_ratio":
+            out["do"] = run_arm(wl, b_do, "do", min(args.micro, 64), arena=arena)
+            out["generated_tok_s_ratio"] = out["pd"]["generated_tok_s"] / out["do"]["generated_tok_s"]
+        print(json.dumps(out))
+    elif args.run == "cfg4":
+        wl = WORKLOADS["cfg4"]
+        if args.decode_steps is not None:
+            wl = wl.with_(steps=args.decode_steps)
+        budget = int((args.budget_gib or 120.0) * GiB)
+        b = max_batch(make_cfg(wl, 1, "pd", args.micro), budget)
+        arena = torch.empty(budget, dtype=torch.uint8, device="cuda")
+        layers = range(wl.L) if args.layers is None else range(args.layers)
+        res = run_arm(wl, b, "pd", args.micro, arena=arena, layers=layers)
+        print(json.dumps({"run": "cfg4", "budget_GiB": budget / GiB, "batch": b, "pd": res}))
+    else:
+        for B, K in CFG5_SWEEP:
+            wl = WORKLOADS["cfg5"].with_(B=B, K=K, name=f"cfg5_B{B}_K{K}")
+            if args.decode_steps is not None:
+                wl = wl.with_(steps=args.decode_steps)
+            res = run_arm(wl, wl.b, "pd", wl.b)
+            print(json.dumps({"run": "cfg5", "block": B, "kv_max": K, "pd": res}), flush=True)
+
+
+if __name__ == "__main__":
+    main()
