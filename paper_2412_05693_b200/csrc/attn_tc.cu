@@ -89,7 +89,27 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   if (!active_b) T[1] = 0;
   const int t_max = active_b ? T[1] : T[0];      // tile B sees at least as many key tiles as tile A
 
-  if (tid == 0) {
+  // The producer warp initialises the barriers and starts the first loads at once; tensor-memory allocation
+  // and the CTA-wide barrier below overlap their latency.
+  auto load_q = [&](int x) {
+    mbar_expect_tx(&bars[B_QFULL + x], L::kTileBytes);
+    for (int c = 0; c < L::kChunks; ++c)
+      tma_load_5d(sm + L::kQ + x * L::kTileBytes + c * 16384, &maps.q, c * 64, 0, kh, i0[x], smp, &bars[B_QFULL + x]);
+  };
+  auto load_kv = [&](int e) {   // ring entry e: K_j for even e, V_j for odd e, j = e / 2
+    const int j = e >> 1, s = e % kKvStages;
+    const bool is_v = e & 1;
+    unsigned char* dst = sm + L::kKV + s * L::kTileBytes;
+    mbar_expect_tx(&bars[B_KVFULL + s], L::kTileBytes);
+    for (int c = 0; c < L::kChunks; ++c) {
+      if (j < t_old)
+        tma_load_3d(dst + c * 16384, is_v ? &maps.v_slab : &maps.k_slab, c * 64, j * kTileN, unit, &bars[B_KVFULL + s]);
+      else
+        tma_load_4d(dst + c * 16384, is_v ? &maps.v_blk : &maps.k_blk, c * 64, kh, (j - t_old) * kTileN, smp,
+                    &bars[B_KVFULL + s]);
+    }
+  };
+  if (warp == 9 && lane == 0) {
     *abort_flag = 0;
     for (int x = 0; x < 2; ++x) {
       mbar_init(&bars[B_QFULL + x], 1);
@@ -99,6 +119,10 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
     }
     for (int s = 0; s < kKvStages; ++s) { mbar_init(&bars[B_KVFULL + s], 1); mbar_init(&bars[B_KVEMPTY + s], 1); }
     mbar_fence_init();
+    load_q(0);
+    load_kv(0);
+    if (active_b) load_q(1);
+    for (int e = 1; e < min(kKvStages, 2 * t_max); ++e) load_kv(e);
   }
   if (warp == 8) tmem_alloc(tmem_slot, kTmemCols);
   tc_fence_before();
@@ -111,24 +135,9 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   if (warp == 9) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      for (int x = 0; x < (active_b ? 2 : 1); ++x) {
-        mbar_expect_tx(&bars[B_QFULL + x], L::kTileBytes);
-        for (int c = 0; c < L::kChunks; ++c)
-          tma_load_5d(sm + L::kQ + x * L::kTileBytes + c * 16384, &maps.q, c * 64, 0, kh, i0[x], smp, &bars[B_QFULL + x]);
-      }
-      for (int e = 0; e < 2 * t_max; ++e) {
-        const int j = e >> 1, s = e % kKvStages;
-        const bool is_v = e & 1;
-        if (e >= kKvStages) mbar_wait(&bars[B_KVEMPTY + s], ((e / kKvStages) - 1) & 1, abort_flag, a.status);
-        unsigned char* dst = sm + L::kKV + s * L::kTileBytes;
-        mbar_expect_tx(&bars[B_KVFULL + s], L::kTileBytes);
-        for (int c = 0; c < L::kChunks; ++c) {
-          if (j < t_old)
-            tma_load_3d(dst + c * 16384, is_v ? &maps.v_slab : &maps.k_slab, c * 64, j * kTileN, unit, &bars[B_KVFULL + s]);
-          else
-            tma_load_4d(dst + c * 16384, is_v ? &maps.v_blk : &maps.k_blk, c * 64, kh, (j - t_old) * kTileN, smp,
-                        &bars[B_KVFULL + s]);
-        }
+      for (int e = kKvStages; e < 2 * t_max; ++e) {
+        mbar_wait(&bars[B_KVEMPTY + e % kKvStages], ((e / kKvStages) - 1) & 1, abort_flag, a.status);
+        load_kv(e);
       }
     }
   } else if (warp == 8) {
@@ -352,12 +361,28 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   const int qt0 = is_old ? 0 : c0 / qpt;           // earlier query tiles cannot see these keys
   const int T = n_qt - qt0;
 
-  if (tid == 0) {
+  auto load_k = [&]() {
+    mbar_expect_tx(&bars[C_KFULL], L::kTileBytes);
+    for (int c = 0; c < L::kChunks; ++c) {
+      if (is_old) tma_load_3d(sm + L::kK + c * 16384, &maps.k_slab, c * 64, kt * kTileN, unit, &bars[C_KFULL]);
+      else tma_load_4d(sm + L::kK + c * 16384, &maps.k_blk, c * 64, kh, c0, smp, &bars[C_KFULL]);
+    }
+  };
+  auto load_q = [&](int t) {
+    const int s = t % kQStages;
+    mbar_expect_tx(&bars[C_QFULL + s], L::kTileBytes);
+    for (int c = 0; c < L::kChunks; ++c)
+      tma_load_5d(sm + L::kQ + s * L::kTileBytes + c * 16384, &maps.q, c * 64, 0, kh, (qt0 + t) * qpt, smp,
+                  &bars[C_QFULL + s]);
+  };
+  if (warp == 9 && lane == 0) {   // barriers and the first loads before the CTA-wide barrier (overlaps TMEM allocation)
     *abort_flag = 0;
     mbar_init(&bars[C_KFULL], 1);
     for (int s = 0; s < kQStages; ++s) { mbar_init(&bars[C_QFULL + s], 1); mbar_init(&bars[C_QEMPTY + s], 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(&bars[C_SFULL + b], 1); mbar_init(&bars[C_SFREE + b], 128); }
     mbar_fence_init();
+    load_k();
+    for (int t = 0; t < min(kQStages, T); ++t) load_q(t);
   }
   if (warp == 8) tmem_alloc(tmem_slot, 256);
   tc_fence_before();
@@ -368,18 +393,9 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
 
   if (warp == 9) {
     if (lane == 0) {
-      mbar_expect_tx(&bars[C_KFULL], L::kTileBytes);
-      for (int c = 0; c < L::kChunks; ++c) {
-        if (is_old) tma_load_3d(sm + L::kK + c * 16384, &maps.k_slab, c * 64, kt * kTileN, unit, &bars[C_KFULL]);
-        else tma_load_4d(sm + L::kK + c * 16384, &maps.k_blk, c * 64, kh, c0, smp, &bars[C_KFULL]);
-      }
-      for (int t = 0; t < T; ++t) {
-        const int s = t % kQStages;
-        if (t >= kQStages) mbar_wait(&bars[C_QEMPTY + s], ((t / kQStages) - 1) & 1, abort_flag, a.status);
-        mbar_expect_tx(&bars[C_QFULL + s], L::kTileBytes);
-        for (int c = 0; c < L::kChunks; ++c)
-          tma_load_5d(sm + L::kQ + s * L::kTileBytes + c * 16384, &maps.q, c * 64, 0, kh, (qt0 + t) * qpt, smp,
-                      &bars[C_QFULL + s]);
+      for (int t = kQStages; t < T; ++t) {
+        mbar_wait(&bars[C_QEMPTY + t % kQStages], ((t / kQStages) - 1) & 1, abort_flag, a.status);
+        load_q(t);
       }
     }
   } else if (warp == 8) {
