@@ -145,27 +145,32 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
     if (lane == 0) {
       const uint32_t idesc_qk = instr_desc(kTileM, kTileN, 0, 0);
       const uint32_t idesc_pv = instr_desc(kTileM, D, 0, 1);  // V is MN-major: d contiguous, keys along K
-      auto kv_addr = [&](int e) { return smem_u32(sm + L::kKV + (e % kKvStages) * L::kTileBytes); };
       auto wait_kv = [&](int e) { mbar_wait(&bars[B_KVFULL + e % kKvStages], (e / kKvStages) & 1, abort_flag, a.status); };
+      // Descriptors differ between MMAs only in the start-address field (low word, 16-byte units), so the
+      // issuing thread adds small constants to precomputed words instead of rebuilding 64-bit descriptors.
+      const uint64_t dk_hi = smem_desc(0, 16, 1024) & 0xffffffff00000000ull;      // K-major operands (Q, K)
+      const uint32_t dk_lo = (uint32_t)(smem_desc(0, 16, 1024) & 0xffffffffull);
+      const uint64_t dv_hi = smem_desc(0, 16384, 1024) & 0xffffffff00000000ull;   // MN-major operand (V)
+      const uint32_t dv_lo = (uint32_t)(smem_desc(0, 16384, 1024) & 0xffffffffull);
+      const uint32_t q_lo[2] = {dk_lo + (smem_u32(sm + L::kQ) >> 4), dk_lo + (smem_u32(sm + L::kQ + L::kTileBytes) >> 4)};
+      const uint32_t kv_lo0 = smem_u32(sm + L::kKV) >> 4;
       auto issue_qk = [&](int x, int j) {   // S_x = Q_x K_j^T
-        const uint32_t q_addr = smem_u32(sm + L::kQ + x * L::kTileBytes), k_addr = kv_addr(2 * j);
+        const uint32_t k_lo = dk_lo + kv_lo0 + ((2 * j) % kKvStages) * (L::kTileBytes >> 4);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
-          const uint64_t da = smem_desc(q_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
-          const uint64_t db = smem_desc(k_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
-          mma_ss(tm_s[x], da, db, idesc_qk, ks > 0 ? 1u : 0u);
+          const uint32_t off = (ks >> 2) * 1024 + (ks & 3) * 2;   // (chunk * 16384 + kstep * 32) / 16
+          mma_ss(tm_s[x], dk_hi | (q_lo[x] + off), dk_hi | (k_lo + off), idesc_qk, ks > 0 ? 1u : 0u);
         }
         mma_commit(&bars[B_SFULL + x]);
       };
       auto issue_pv = [&](int x, int j) {   // O_x += P_x V_j, P_x read from tensor memory (over S_x)
         mbar_wait(&bars[B_PFULL + x], j & 1, abort_flag, a.status);
         tc_fence_after();
-        const uint32_t v_addr = kv_addr(2 * j + 1);
+        const uint32_t v_lo = dv_lo + kv_lo0 + ((2 * j + 1) % kKvStages) * (L::kTileBytes >> 4);
+        const uint32_t acc0 = j > 0 ? 1u : 0u;
 #pragma unroll
-        for (int ks = 0; ks < kTileN / 16; ++ks) {
-          const uint64_t db = smem_desc(v_addr + ks * 2048, 16384, 1024);
-          mma_ts(tm_o[x], tm_s[x] + ks * 8, db, idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
-        }
+        for (int ks = 0; ks < kTileN / 16; ++ks)   // 16 keys = 2 row groups of 1024 bytes per step
+          mma_ts(tm_o[x], tm_s[x] + ks * 8, dv_hi | (v_lo + ks * 128), idesc_pv, ks > 0 ? 1u : acc0);
         mma_commit(&bars[B_ODONE + x]);
       };
       mbar_wait(&bars[B_QFULL + 0], 0, abort_flag, a.status);
@@ -401,19 +406,21 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   } else if (warp == 8) {
     if (lane == 0) {
       const uint32_t idesc = instr_desc(kTileN, kTileM, 0, 0);
-      const uint32_t k_addr = smem_u32(sm + L::kK);
+      const uint64_t d_hi = smem_desc(0, 16, 1024) & 0xffffffff00000000ull;
+      const uint32_t d_lo = (uint32_t)(smem_desc(0, 16, 1024) & 0xffffffffull);
+      const uint32_t k_lo = d_lo + (smem_u32(sm + L::kK) >> 4);
       mbar_wait(&bars[C_KFULL], 0, abort_flag, a.status);
       for (int t = 0; t < T; ++t) {
         const int s = t % kQStages, b = t & 1;
         mbar_wait(&bars[C_QFULL + s], (t / kQStages) & 1, abort_flag, a.status);
         if (t >= 2) mbar_wait(&bars[C_SFREE + b], ((t >> 1) - 1) & 1, abort_flag, a.status);
         tc_fence_after();
-        const uint32_t q_addr = smem_u32(sm + L::kQ + s * L::kTileBytes);
+        const uint32_t q_lo = d_lo + ((smem_u32(sm + L::kQ) >> 4) + s * (L::kTileBytes >> 4));
+        const uint32_t ts = b ? tmem + 128 : tmem;
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint64_t da = smem_desc(k_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
-          const uint64_t db = smem_desc(q_addr + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024);
-          mma_ss(tm_s[b], da, db, idesc, ks > 0 ? 1u : 0u);
+        for (int ks = 0; ks < D / 16; ++ks) {   // only the start-address word of the descriptors changes
+          const uint32_t off = (ks >> 2) * 1024 + (ks & 3) * 2;
+          mma_ss(ts, d_hi | (k_lo + off), d_hi | (q_lo + off), idesc, ks > 0 ? 1u : 0u);
         }
         mma_commit(&bars[C_SFULL + b]);
         mma_commit(&bars[C_QEMPTY + s]);
