@@ -323,9 +323,11 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
 
 // ------------------------------------------------------------------------------------------------------
 // Score pass.  CTA = (tile of 128 candidate keys, unit).  A = the key tile (loaded once), B = the unit's query
-// tiles streamed through a ring; S^T lands in TMEM with lane = key, column = query row.  Two reducer
-// warpgroups take alternate query tiles (one TMEM buffer each); their partial sums are added in a fixed order.
-constexpr int kScoreThreads = 320;   // warps 0-3, 4-7: reducers; warp 8: MMA + TMEM owner; warp 9: TMA
+// tiles streamed through a ring; S^T lands in TMEM with lane = key, column = query row.  The pass is bound by
+// one exponential per visible pair, so four reducer warpgroups (one TMEM buffer each, query tiles taken round
+// robin) keep the special-function units busy; their partial sums are added in a fixed order.
+constexpr int kScoreWG = 4;                              // reducer warpgroups == TMEM buffers of 128 columns
+constexpr int kScoreThreads = 128 * kScoreWG + 64;       // + warp 4*WG: MMA + TMEM owner, warp 4*WG+1: TMA
 constexpr int kQStages = 3;
 
 template <int D>
@@ -334,18 +336,19 @@ struct ScoreSmem {
   static constexpr int kTileBytes = kChunks * 16384;
   static constexpr int kK = 0;
   static constexpr int kQ = kK + kTileBytes;
-  static constexpr int kLse = kQ + kQStages * kTileBytes;      // 2 x 128 floats
-  static constexpr int kPart = kLse + 2 * 128 * 4;             // 128 floats: warpgroup 1's partial sums
-  static constexpr int kBars = kPart + 128 * 4;
+  static constexpr int kLse = kQ + kQStages * kTileBytes;      // [WG][128] floats
+  static constexpr int kPart = kLse + kScoreWG * 128 * 4;      // [WG][128] floats: partial sums
+  static constexpr int kBars = kPart + kScoreWG * 128 * 4;
   static constexpr int kTotal = kBars + 256 + 1024;
 };
-enum { C_KFULL = 0, C_QFULL = 1, C_QEMPTY = C_QFULL + kQStages, C_SFULL = C_QEMPTY + kQStages, C_SFREE = C_SFULL + 2,
-       C_COUNT = C_SFREE + 2 };
+enum { C_KFULL = 0, C_QFULL = 1, C_QEMPTY = C_QFULL + kQStages, C_SFULL = C_QEMPTY + kQStages,
+       C_SFREE = C_SFULL + kScoreWG, C_COUNT = C_SFREE + kScoreWG };
 
 template <int D>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   using L = ScoreSmem<D>;
+  constexpr int kMmaWarp = 4 * kScoreWG, kTmaWarp = 4 * kScoreWG + 1;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::kBars);
@@ -380,30 +383,29 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
       tma_load_5d(sm + L::kQ + s * L::kTileBytes + c * 16384, &maps.q, c * 64, 0, kh, (qt0 + t) * qpt, smp,
                   &bars[C_QFULL + s]);
   };
-  if (warp == 9 && lane == 0) {   // barriers and the first loads before the CTA-wide barrier (overlaps TMEM allocation)
+  if (warp == kTmaWarp && lane == 0) {   // barriers and the first loads before the CTA-wide barrier (overlaps TMEM allocation)
     *abort_flag = 0;
     mbar_init(&bars[C_KFULL], 1);
     for (int s = 0; s < kQStages; ++s) { mbar_init(&bars[C_QFULL + s], 1); mbar_init(&bars[C_QEMPTY + s], 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(&bars[C_SFULL + b], 1); mbar_init(&bars[C_SFREE + b], 128); }
+    for (int b = 0; b < kScoreWG; ++b) { mbar_init(&bars[C_SFULL + b], 1); mbar_init(&bars[C_SFREE + b], 128); }
     mbar_fence_init();
     load_k();
     for (int t = 0; t < min(kQStages, T); ++t) load_q(t);
   }
-  if (warp == 8) tmem_alloc(tmem_slot, 256);
+  if (warp == kMmaWarp) tmem_alloc(tmem_slot, 128 * kScoreWG);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tm_s[2] = {tmem, tmem + 128};
 
-  if (warp == 9) {
+  if (warp == kTmaWarp) {
     if (lane == 0) {
       for (int t = kQStages; t < T; ++t) {
         mbar_wait(&bars[C_QEMPTY + t % kQStages], ((t / kQStages) - 1) & 1, abort_flag, a.status);
         load_q(t);
       }
     }
-  } else if (warp == 8) {
+  } else if (warp == kMmaWarp) {
     if (lane == 0) {
       const uint32_t idesc = instr_desc(kTileN, kTileM, 0, 0);
       const uint64_t d_hi = smem_desc(0, 16, 1024) & 0xffffffff00000000ull;
@@ -411,12 +413,12 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
       const uint32_t k_lo = d_lo + (smem_u32(sm + L::kK) >> 4);
       mbar_wait(&bars[C_KFULL], 0, abort_flag, a.status);
       for (int t = 0; t < T; ++t) {
-        const int s = t % kQStages, b = t & 1;
+        const int s = t % kQStages, b = t % kScoreWG;
         mbar_wait(&bars[C_QFULL + s], (t / kQStages) & 1, abort_flag, a.status);
-        if (t >= 2) mbar_wait(&bars[C_SFREE + b], ((t >> 1) - 1) & 1, abort_flag, a.status);
+        if (t >= kScoreWG) mbar_wait(&bars[C_SFREE + b], ((t / kScoreWG) - 1) & 1, abort_flag, a.status);
         tc_fence_after();
         const uint32_t q_lo = d_lo + ((smem_u32(sm + L::kQ) >> 4) + s * (L::kTileBytes >> 4));
-        const uint32_t ts = b ? tmem + 128 : tmem;
+        const uint32_t ts = tmem + b * 128;
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {   // only the start-address word of the descriptors changes
           const uint32_t off = (ks >> 2) * 1024 + (ks & 3) * 2;
@@ -427,12 +429,13 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
       }
     }
   } else {
-    const int wg = warp >> 2;                      // reducer warpgroup: takes query tiles t = wg, wg + 2, ...
+    const int wg = warp >> 2;                      // reducer warpgroup: takes query tiles t = wg, wg + WG, ...
     const int quad = warp & 3;
     const int key = quad * 32 + lane;              // key inside the tile == TMEM lane
-    const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
+    const uint32_t ts = tmem + wg * 128 + ((uint32_t)(quad * 32) << 16);
+    const float* lse_w = sLse + wg * 128;
     float acc = 0.f;
-    for (int t = wg; t < T; t += 2) {
+    for (int t = wg; t < T; t += kScoreWG) {
       const int qrow0 = (qt0 + t) * kTileM;
       // this tile's log2-sum-exp values; +inf for rows past the block's end (weight 0)
       {
@@ -440,47 +443,55 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
         sLse[wg * 128 + key] = rr < R ? a.lse2[(size_t)unit * R + rr] : INFINITY;
       }
       named_bar_sync(1 + wg, 128);
-      mbar_wait(&bars[C_SFULL + wg], (t >> 1) & 1, abort_flag, a.status);
+      mbar_wait(&bars[C_SFULL + wg], (t / kScoreWG) & 1, abort_flag, a.status);
       tc_fence_after();
       // first query row of the tile that may see this key (causal mask inside the block)
       const int first_vis = is_old ? 0 : max(0, (c0 + key) * a.g - qrow0);
-      float part = 0.f;
+      const bool nomask = __all_sync(0xffffffffu, first_vis == 0);
+      float p0 = 0.f, p1 = 0.f;
+      uint32_t cur[32], nxt[32];
+      tmem_ld32(ts, cur);
+      tmem_wait_ld();
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t ra[32], rb[32];
-        tmem_ld32(tm_s[wg] + lane_addr + half * 64, ra);
-        tmem_ld32(tm_s[wg] + lane_addr + half * 64 + 32, rb);
-        tmem_wait_ld();
+      for (int cc = 0; cc < 4; ++cc) {
+        if (cc < 3) tmem_ld32(ts + (cc + 1) * 32, nxt);   // next chunk loads while this one is used
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int col = half * 64 + e;
-          const float p = ex2(fmaf(__uint_as_float(ra[e]), a.scale_log2, -sLse[wg * 128 + col]));
-          part += col >= first_vis ? p : 0.f;
+        for (int e = 0; e < 32; e += 2) {
+          const int col = cc * 32 + e;
+          float e0 = ex2(fmaf(__uint_as_float(cur[e]), a.scale_log2, -lse_w[col]));
+          float e1 = ex2(fmaf(__uint_as_float(cur[e + 1]), a.scale_log2, -lse_w[col + 1]));
+          if (!nomask) {
+            e0 = col >= first_vis ? e0 : 0.f;
+            e1 = col + 1 >= first_vis ? e1 : 0.f;
+          }
+          p0 += e0;
+          p1 += e1;
         }
+        if (cc < 3) {
+          tmem_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const int col = half * 64 + 32 + e;
-          const float p = ex2(fmaf(__uint_as_float(rb[e]), a.scale_log2, -sLse[wg * 128 + col]));
-          part += col >= first_vis ? p : 0.f;
+          for (int e = 0; e < 32; ++e) cur[e] = nxt[e];
         }
       }
-      acc += part;
+      acc += p0 + p1;
       tc_fence_before();
       mbar_arrive(&bars[C_SFREE + wg]);
       named_bar_sync(1 + wg, 128);                 // everyone is done with this tile's sLse before it is rewritten
     }
-    if (wg == 1) sPart[key] = acc;
-    named_bar_sync(3, 256);
+    sPart[wg * 128 + key] = acc;
+    named_bar_sync(1 + kScoreWG, 128 * kScoreWG);
     if (wg == 0) {
-      acc += sPart[key];
+      float tot = 0.f;
+#pragma unroll
+      for (int w = 0; w < kScoreWG; ++w) tot += sPart[w * 128 + key];   // fixed order
       const int j = is_old ? kt * kTileN + key : c0 + key;
-      if (is_old) { if (j < a.n_old) a.sum_weights[(size_t)unit * a.cap + j] += acc; }
-      else if (j < a.I) a.new_sum[(size_t)unit * a.I + j] = acc;
+      if (is_old) { if (j < a.n_old) a.sum_weights[(size_t)unit * a.cap + j] += tot; }
+      else if (j < a.I) a.new_sum[(size_t)unit * a.I + j] = tot;
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) tmem_dealloc(tmem, 256);
+  if (warp == kMmaWarp) tmem_dealloc(tmem, 128 * kScoreWG);
 }
 
 // ------------------------------------------------------------------------------------------------------
