@@ -186,6 +186,13 @@ bm_status_t bm_cache_set_len(bm_cache_t* cache, int32_t layer, int32_t sample, i
  * up a bounded wait (its results are then undefined; the context stays usable). */
 bm_status_t bm_cache_status(bm_cache_t* cache, int32_t* device_status /*HOST out*/, void* cuda_stream);
 
+/* Reset the device status word to BM_OK (stream-ordered). */
+bm_status_t bm_cache_clear_status(bm_cache_t* cache, void* cuda_stream);
+/* Failure-detection self-test (the paper has no counterpart): enqueue a one-warp kernel whose bounded wait can
+ * never be satisfied.  It gives up after its poll limit, writes BM_ERR_TIMEOUT to the status word and ends
+ * normally; bm_cache_status then reports BM_ERR_TIMEOUT and the context stays usable.  Nothing else is touched. */
+bm_status_t bm_selftest_wait_timeout(bm_cache_t* cache, void* cuda_stream);
+
 /* ---- per-kernel timing (measurement aid; the paper has no counterpart) ----
  * While enabled, every kernel launch of this library is bracketed by two CUDA events on its stream.
  * bm_profile_read waits for the recorded launches of one kernel class, returns their summed duration in

@@ -55,6 +55,8 @@ SIGNATURES = {
     "bm_cache_import": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp]),
     "bm_cache_set_len": (_i32, [_vp, _i32, _i32, _i32, _i32]),
     "bm_cache_status": (_i32, [_vp, C.POINTER(_i32), _vp]),
+    "bm_cache_clear_status": (_i32, [_vp, _vp]),
+    "bm_selftest_wait_timeout": (_i32, [_vp, _vp]),
     "bm_profile_enable": (_i32, [_i32]),
     "bm_profile_read": (_i32, [_i32, C.POINTER(C.c_float), C.POINTER(_i32)]),
     "bm_kernel_launch_count": (C.c_uint64, []),
@@ -301,6 +303,13 @@ class BatchMaxCache:
         _check(lib().bm_cache_import(self.h, layer, sample, kv_head, _ptr(ids.contiguous()), _ptr(sw.contiguous()),
                                      _ptr(kr.contiguous()), _ptr(vr.contiguous()), ids.shape[0], _stream(stream)),
                "bm_cache_import")
+
+    def clear_status(self, stream=None):
+        _check(lib().bm_cache_clear_status(self.h, _stream(stream)), "bm_cache_clear_status")
+
+    def selftest_wait_timeout(self, stream=None):
+        """Enqueue the bounded-wait self-test: afterwards status() reports 6 (BM_ERR_TIMEOUT)."""
+        _check(lib().bm_selftest_wait_timeout(self.h, _stream(stream)), "bm_selftest_wait_timeout")
 
     def status(self, stream=None) -> int:
         w = _i32(0)

@@ -477,6 +477,22 @@ bm_status_t bm_cache_status(bm_cache_t* c, int32_t* device_status, void* cuda_st
   return BM_OK;
 }
 
+bm_status_t bm_cache_clear_status(bm_cache_t* c, void* cuda_stream) {
+  if (c == nullptr) return BM_ERR_INVALID;
+  bm_status_t s = set_device(c);
+  if (s != BM_OK) return s;
+  return cudaMemsetAsync(c->status, 0, sizeof(int32_t), static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? BM_OK : BM_ERR_CUDA;
+}
+
+bm_status_t bm_selftest_wait_timeout(bm_cache_t* c, void* cuda_stream) {
+  if (c == nullptr) return BM_ERR_INVALID;
+  bm_status_t s = set_device(c);
+  if (s != BM_OK) return s;
+  return launch_wait_timeout_selftest(c->status, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+             ? BM_OK : BM_ERR_CUDA;
+}
+
 bm_status_t bm_profile_enable(int32_t on) {
   g_profile_on = on != 0;
   return BM_OK;

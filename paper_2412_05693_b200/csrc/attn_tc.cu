@@ -595,7 +595,23 @@ cudaError_t launch_score_t(const CacheView& c, const BlockArgs& a, cudaStream_t 
   return cudaGetLastError();
 }
 
+// Self-test of the bounded wait: one thread waits on a barrier that nothing ever arrives on.  The wait gives up
+// after its poll limit, records BM_ERR_TIMEOUT in the status word and the kernel ends normally.
+__global__ void wait_timeout_selftest(int* status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) { abort_flag = 0; mbar_init(&bar, 1); mbar_fence_init(); }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(&bar, 0, &abort_flag, status, 1 << 16);
+}
+
 }  // namespace
+
+cudaError_t launch_wait_timeout_selftest(int* status, cudaStream_t st) {
+  wait_timeout_selftest<<<1, 32, 0, st>>>(status);
+  count_launch();
+  return cudaGetLastError();
+}
 
 bool tc_path_available() { return encode_fn() != nullptr; }
 

@@ -55,6 +55,7 @@ size_t decode_mma_smem_bytes(int d, int g, int n_rows, int target);
 size_t evict_smem_bytes(int n_cand, int target);
 size_t decode_smem_bytes(int d, int g, int n_rows, int target);
 bool tc_path_available();
+cudaError_t launch_wait_timeout_selftest(int* status, cudaStream_t st);
 cudaError_t launch_attn_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used);
 cudaError_t launch_score_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used);
 

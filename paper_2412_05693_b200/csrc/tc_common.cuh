@@ -29,10 +29,11 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* b) {
 // BM_ERR_TIMEOUT in the device status word and raises the CTA's abort flag; once the flag is up every
 // later wait returns at once, so the kernel runs to its normal end (TMEM release included) with
 // undefined results instead of hanging.
-__device__ __forceinline__ void mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ void mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag, int* status,
+                                          int limit = kWaitLimit) {
   if (*abort_flag) return;
   const uint32_t addr = smem_u32(b);
-  for (int it = 0; it < kWaitLimit; ++it) {
+  for (int it = 0; it < limit; ++it) {
     uint32_t ok;
     asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}\n"
                  : "=r"(ok) : "r"(addr), "r"(parity) : "memory");

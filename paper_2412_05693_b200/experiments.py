@@ -37,10 +37,14 @@ def peaks():
     return 6650.0, 1400.0, "fallback"
 
 
+DECODE_MICRO = 2048   # samples per decode call (decode inputs are tiny, so ranges can be much wider than in prefill)
+
+
 def make_cfg(wl: Workload, batch: int, arm: str, micro: int, device: int = 0) -> Config:
     growth = max(1, wl.p_dec) if arm == "pd" else wl.s + max(1, wl.p_dec) - wl.K
     return Config(batch=batch, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.d, kv_max=wl.K, block_max=wl.B,
-                  growth=growth, dtype=wl.dtype, n_layers=wl.L, device=device, max_call_samples=micro)
+                  growth=growth, dtype=wl.dtype, n_layers=wl.L, device=device,
+                  max_call_samples=max(micro, min(batch, DECODE_MICRO)))
 
 
 class Timer:
@@ -78,7 +82,8 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
     ms_pre = ms_dec = 0.0
     layers = range(wl.L) if layers is None else layers
     out_blk = torch.empty(micro, wl.B, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
-    out_dec = torch.empty(micro, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
+    micro_dec = max(micro, min(batch, DECODE_MICRO))
+    out_dec = torch.empty(micro_dec, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
     pairs = 0
     for layer in layers:
         n = 0
@@ -102,8 +107,8 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
         for t in range(wl.steps):
             full = n + 1 >= wl.K + wl.p_dec
             ev = wl.K if full else -1
-            for s0 in range(0, batch, micro):
-                ns = min(micro, batch - s0)
+            for s0 in range(0, batch, micro_dec):
+                ns = min(micro_dec, batch - s0)
                 q, k, v = inp.block(layer, wl.s + t, 1, s0, ns)
                 q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
                 t_dec(lambda: cache.decode_step(q, k, v, out=out_dec[:ns], evict_to=ev, layer=layer, sample0=s0))
@@ -121,6 +126,7 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
     dec_bytes = batch * wl.Hkv * n_layers * wl.steps * (n1 * (2 * wl.d * e + 16) + 2 * wl.d * e + 2 * wl.g * wl.d * e)
     res = {
         "workload": wl.name, "arm": arm, "batch": batch, "layers_run": n_layers, "micro_batch": micro,
+        "decode_micro_batch": micro_dec,
         "arena_GiB": need / GiB, "final_n": n_end, "final_curr_id": cur,
         "prefill_ms": ms_pre, "decode_ms": ms_dec,
         "prefill_tok_s": batch * wl.s * n_layers / (ms_pre * 1e-3),

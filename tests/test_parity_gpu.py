@@ -136,6 +136,21 @@ def test_error_codes_and_state_tracking():
     cache.close()
 
 
+def test_bounded_wait_times_out_and_context_survives():
+    # failure detection without a GPU fault: a wait that nothing satisfies gives up, the status word says so,
+    # and the same handle keeps working afterwards
+    wl = tiny("timeout", dtype="bf16", d=128, Hq=8, Hkv=2, s=96, B=48, K=40, steps=0)
+    cache = bm.BatchMaxCache(make_config(wl))
+    assert cache.status() == 0
+    cache.selftest_wait_timeout()
+    assert cache.status() == 6                     # BM_ERR_TIMEOUT
+    cache.clear_status()
+    assert cache.status() == 0
+    cache.close()
+    st = run_lockstep(wl, all_units(wl), check_rows_every=1)
+    assert st["calls"] == 2
+
+
 def run_free(wl, host=False, micro=None):
     """Whole schedule on the GPU only; returns final state and all outputs (for determinism / variants)."""
     cfg = make_config(wl)
