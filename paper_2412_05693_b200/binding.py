@@ -254,11 +254,14 @@ class BatchMaxCache:
 
     # -- host-fed variants ---------------------------------------------------------------------------
     def _stage(self, ns, I):
+        """Two staging buffers used alternately, so that consecutive host-fed calls overlap their copies."""
         need = staging_bytes(self.cfg, ns, I)
-        if self._staging is None or self._staging.numel() < need:
-            self._staging = self.torch.empty(need, dtype=self.torch.uint8,
-                                             device=self.torch.device("cuda", self.cfg.device))
-        return self._staging
+        if self._staging is None or self._staging[0].numel() < need:
+            dev = self.torch.device("cuda", self.cfg.device)
+            self._staging = [self.torch.empty(need, dtype=self.torch.uint8, device=dev) for _ in range(2)]
+            self._stage_turn = 0
+        self._stage_turn ^= 1
+        return self._staging[self._stage_turn]
 
     def prefill_block_host(self, q, k, v, pos0: int, out, evict_to: int = -1, layer: int = 0, sample0: int = 0,
                            stream=None):

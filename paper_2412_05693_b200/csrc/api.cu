@@ -97,6 +97,12 @@ struct bm_cache {
   float* ws_lse;
   float* ws_new_sum;
   std::vector<int32_t> n, curr_id;  // [L * b] host mirror
+  // host-fed calls: inputs are copied on an internal stream so that the copy of one call overlaps the
+  // compute and the output copy of the previous one; two staging buffers can be in flight
+  cudaStream_t in_stream = nullptr;
+  struct Slot { void* staging = nullptr; cudaEvent_t in_done = nullptr; cudaEvent_t call_done = nullptr; };
+  Slot slots[2];
+  int next_slot = 0;
 };
 
 namespace {
@@ -218,6 +224,15 @@ bm_status_t bm_cache_create(const bm_config_t* cfg, void* arena, size_t arena_by
 
 bm_status_t bm_cache_destroy(bm_cache_t* cache) {
   if (cache == nullptr) return BM_ERR_INVALID;
+  if (cache->in_stream != nullptr) {
+    cudaSetDevice(cache->cfg.device);
+    cudaStreamSynchronize(cache->in_stream);
+    for (auto& sl : cache->slots) {
+      if (sl.in_done) cudaEventDestroy(sl.in_done);
+      if (sl.call_done) cudaEventDestroy(sl.call_done);
+    }
+    cudaStreamDestroy(cache->in_stream);
+  }
   delete cache;
   return BM_OK;
 }
@@ -368,14 +383,41 @@ static bm_status_t host_pass(bm_cache_t* c, int layer, int sample0, int nsamples
   if ((s = set_device(c)) != BM_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   char* sp = static_cast<char*>(staging);
-  if (cudaMemcpyAsync(sp + oq, q, qb, cudaMemcpyHostToDevice, st) != cudaSuccess) return BM_ERR_CUDA;
-  if (cudaMemcpyAsync(sp + ok, k, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return BM_ERR_CUDA;
-  if (cudaMemcpyAsync(sp + ov, v, kb, cudaMemcpyHostToDevice, st) != cudaSuccess) return BM_ERR_CUDA;
+  // Inputs go over an internal stream unless cuda_stream is being captured into a graph.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  cudaStreamIsCapturing(st, &cap);
+  bm_cache::Slot* slot = nullptr;
+  cudaStream_t in = st;
+  if (cap == cudaStreamCaptureStatusNone) {
+    if (c->in_stream == nullptr) {
+      if (cudaStreamCreateWithFlags(&c->in_stream, cudaStreamNonBlocking) != cudaSuccess) return BM_ERR_CUDA;
+      for (auto& sl : c->slots) {
+        if (cudaEventCreateWithFlags(&sl.in_done, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&sl.call_done, cudaEventDisableTiming) != cudaSuccess)
+          return BM_ERR_CUDA;
+      }
+    }
+    for (auto& sl : c->slots)
+      if (sl.staging == staging) slot = &sl;
+    if (slot == nullptr) { slot = &c->slots[c->next_slot]; c->next_slot ^= 1; }
+    in = c->in_stream;
+    // the staging buffer is free again once the previous call that used this slot has finished with it
+    if (slot->staging != nullptr && cudaStreamWaitEvent(in, slot->call_done, 0) != cudaSuccess) return BM_ERR_CUDA;
+    slot->staging = staging;
+  }
+  if (cudaMemcpyAsync(sp + oq, q, qb, cudaMemcpyHostToDevice, in) != cudaSuccess) return BM_ERR_CUDA;
+  if (cudaMemcpyAsync(sp + ok, k, kb, cudaMemcpyHostToDevice, in) != cudaSuccess) return BM_ERR_CUDA;
+  if (cudaMemcpyAsync(sp + ov, v, kb, cudaMemcpyHostToDevice, in) != cudaSuccess) return BM_ERR_CUDA;
+  if (slot != nullptr) {
+    if (cudaEventRecord(slot->in_done, in) != cudaSuccess) return BM_ERR_CUDA;
+    if (cudaStreamWaitEvent(st, slot->in_done, 0) != cudaSuccess) return BM_ERR_CUDA;
+  }
   s = decode ? bm_decode_step(c, layer, sample0, nsamples, sp + oq, sp + ok, sp + ov, sp + oo, evict_to, cuda_stream)
              : bm_prefill_block(c, layer, sample0, nsamples, sp + oq, sp + ok, sp + ov, I, pos0, sp + oo, evict_to,
                                 cuda_stream);
   if (s != BM_OK) return s;
   if (cudaMemcpyAsync(out, sp + oo, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return BM_ERR_CUDA;
+  if (slot != nullptr && cudaEventRecord(slot->call_done, st) != cudaSuccess) return BM_ERR_CUDA;
   return BM_OK;
 }
 
