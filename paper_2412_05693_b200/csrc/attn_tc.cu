@@ -9,6 +9,8 @@
 //                 in a fixed order (deterministic, no atomics).
 // Query rows of a unit are ordered r = i * g + h (input i, head h of the group), so a tile of 128 rows shares
 // its K/V tiles among the g heads of the group.
+#include <cstdlib>
+
 #include "tc_common.cuh"
 #include "common.cuh"
 
@@ -42,30 +44,33 @@ struct TcArgs {
 };
 
 // ------------------------------------------------------------------------------------------------------
-// Forward.  Warps 0-3: softmax of tile A, warps 4-7: softmax of tile B, warp 8: MMA issue + TMEM owner,
-// warp 9: TMA producer.  TMEM: S_A | S_B (fp32 logits, overwritten in place by the bf16 probabilities that
-// feed P.V as the tensor-memory operand) | O_A | O_B.
-constexpr int kFwdThreads = 320;
-constexpr int kKvStages = 4;     // ring of K/V tiles: entry 2j = K_j, entry 2j+1 = V_j
-constexpr int kTmemCols = 512;
-
-template <int D>
+// Forward, NT query tiles per CTA.  NT = 2 (large grids): warps 0-3 / 4-7 are the softmax warpgroups of tiles A / B,
+// warp 8 issues the MMAs and owns the tensor memory, warp 9 is the TMA producer; one CTA per SM, both tiles share
+// every K/V tile.  NT = 1 (small grids): four softmax warps + MMA warp + TMA warp, half the shared and tensor
+// memory, two CTAs per SM, so that one CTA's prologue and epilogue overlap the other's main loop.
+// TMEM: S tiles (fp32 logits, overwritten in place by the bf16 probabilities that feed P.V as the tensor-memory
+// operand), then the O accumulators.
+template <int D, int NT>
 struct FwdSmem {
+  static constexpr int kStages = NT == 2 ? 4 : 2;        // ring of K/V tiles: entry 2j = K_j, entry 2j+1 = V_j
   static constexpr int kChunks = D / 64;                 // 64-element (128-byte) column chunks per row
   static constexpr int kTileBytes = kChunks * 16384;     // 128 rows x D bf16
-  static constexpr int kQ = 0;                           // two query tiles (reused to stage the outputs)
-  static constexpr int kKV = kQ + 2 * kTileBytes;
-  static constexpr int kBars = kKV + kKvStages * kTileBytes;
+  static constexpr int kQ = 0;                           // query tiles (reused to stage the outputs)
+  static constexpr int kKV = kQ + NT * kTileBytes;
+  static constexpr int kBars = kKV + kStages * kTileBytes;
   static constexpr int kTotal = kBars + 256 + 1024;      // + barriers + alignment slack
+  static constexpr int kThreads = 128 * NT + 64;
 };
 
-enum { B_QFULL = 0, B_KVFULL = 2, B_KVEMPTY = B_KVFULL + kKvStages, B_SFULL = B_KVEMPTY + kKvStages,
-       B_PFULL = B_SFULL + 2, B_ODONE = B_PFULL + 2, B_COUNT = B_ODONE + 2 };
-
-template <int D>
-__global__ void __launch_bounds__(kFwdThreads, 1)
+template <int D, int NT>
+__global__ void __launch_bounds__(128 * NT + 64, NT == 2 ? 1 : 2)
 attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
-  using L = FwdSmem<D>;
+  using L = FwdSmem<D, NT>;
+  constexpr int kKvStages = L::kStages;
+  constexpr int kMmaWarp = 4 * NT, kTmaWarp = 4 * NT + 1;
+  constexpr int kTmemCols = 256 * NT;
+  constexpr int B_QFULL = 0, B_KVFULL = 2, B_KVEMPTY = B_KVFULL + kKvStages, B_SFULL = B_KVEMPTY + kKvStages,
+                B_PFULL = B_SFULL + 2, B_ODONE = B_PFULL + 2, B_COUNT = B_ODONE + 2;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::kBars);
@@ -80,12 +85,12 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   int row0[2], i0[2], T[2];
 #pragma unroll
   for (int x = 0; x < 2; ++x) {
-    row0[x] = (blockIdx.x * 2 + x) * kTileM;
-    i0[x] = (blockIdx.x * 2 + x) * qpt;
+    row0[x] = (blockIdx.x * NT + x) * kTileM;
+    i0[x] = (blockIdx.x * NT + x) * qpt;
     const int i_last = min(a.I - 1, i0[x] + qpt - 1);
     T[x] = t_old + i_last / kTileN + 1;          // cached-key tiles + block-key tiles up to the tile's last input
   }
-  const bool active_b = row0[1] < R;
+  const bool active_b = NT == 2 && row0[1] < R;
   if (!active_b) T[1] = 0;
   const int t_max = active_b ? T[1] : T[0];      // tile B sees at least as many key tiles as tile A
 
@@ -109,7 +114,7 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
                     &bars[B_KVFULL + s]);
     }
   };
-  if (warp == 9 && lane == 0) {
+  if (warp == kTmaWarp && lane == 0) {
     *abort_flag = 0;
     for (int x = 0; x < 2; ++x) {
       mbar_init(&bars[B_QFULL + x], 1);
@@ -124,15 +129,15 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
     if (active_b) load_q(1);
     for (int e = 1; e < min(kKvStages, 2 * t_max); ++e) load_kv(e);
   }
-  if (warp == 8) tmem_alloc(tmem_slot, kTmemCols);
+  if (warp == kMmaWarp) tmem_alloc(tmem_slot, kTmemCols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tm_s[2] = {tmem, tmem + 128};
-  const uint32_t tm_o[2] = {tmem + 256, tmem + 384};
+  const uint32_t tm_o[2] = {tmem + 128 * NT, tmem + 128 * NT + 128};
 
-  if (warp == 9) {
+  if (warp == kTmaWarp) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       for (int e = kKvStages; e < 2 * t_max; ++e) {
@@ -140,7 +145,7 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
         load_kv(e);
       }
     }
-  } else if (warp == 8) {
+  } else if (warp == kMmaWarp) {
     // ------------------------------------------------------------------ MMA issuer (one thread)
     if (lane == 0) {
       const uint32_t idesc_qk = instr_desc(kTileM, kTileN, 0, 0);
@@ -318,7 +323,7 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) tmem_dealloc(tmem, kTmemCols);
+  if (warp == kMmaWarp) tmem_dealloc(tmem, kTmemCols);
 }
 
 // ------------------------------------------------------------------------------------------------------
@@ -563,20 +568,31 @@ TcArgs make_args(const CacheView& c, const BlockArgs& a) {
 TcMaps g_maps;
 const void* g_maps_q = nullptr;
 
-template <int D>
-cudaError_t launch_fwd_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+template <int D, int NT>
+cudaError_t launch_fwd_nt(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+  using L = FwdSmem<D, NT>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kTotal);
+    cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc<D, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   const int R = a.I * c.g;
-  dim3 grid((R + 2 * kTileM - 1) / (2 * kTileM), c.nsamples * c.Hkv);
+  dim3 grid((R + NT * kTileM - 1) / (NT * kTileM), c.nsamples * c.Hkv);
   ProfileScope prof(kAttnFwd, st);
-  attn_fwd_tc<D><<<grid, kFwdThreads, FwdSmem<D>::kTotal, st>>>(g_maps, make_args(c, a));
+  attn_fwd_tc<D, NT><<<grid, L::kThreads, L::kTotal, st>>>(g_maps, make_args(c, a));
   count_launch();
   return cudaGetLastError();
+}
+
+// One query tile per CTA with two CTAs per SM measured faster than two tiles per CTA on every shape tried
+// (cfg2: 530 vs 507 TFLOP/s, cfg3 shape at b=256: 789 vs 776): overlapping one CTA's first loads and epilogue
+// with the other's main loop is worth more than sharing K/V tiles.  BM_FWD_TILES=2 selects the other variant.
+int g_fwd_tiles_override = 0;
+
+template <int D>
+cudaError_t launch_fwd_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+  return g_fwd_tiles_override == 2 ? launch_fwd_nt<D, 2>(c, a, st) : launch_fwd_nt<D, 1>(c, a, st);
 }
 
 template <int D>
@@ -613,7 +629,15 @@ cudaError_t launch_wait_timeout_selftest(int* status, cudaStream_t st) {
   return cudaGetLastError();
 }
 
-bool tc_path_available() { return encode_fn() != nullptr; }
+bool tc_path_available() {
+  static bool init = false;
+  if (!init) {
+    init = true;
+    const char* e = std::getenv("BM_FWD_TILES");
+    if (e != nullptr) g_fwd_tiles_override = std::atoi(e);
+  }
+  return encode_fn() != nullptr;
+}
 
 cudaError_t launch_attn_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used) {
   *used = 0;
