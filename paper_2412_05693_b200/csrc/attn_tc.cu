@@ -331,9 +331,9 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
 // tiles streamed through a ring; S^T lands in TMEM with lane = key, column = query row.  The pass is bound by
 // one exponential per visible pair, so four reducer warpgroups (one TMEM buffer each, query tiles taken round
 // robin) keep the special-function units busy; their partial sums are added in a fixed order.
-constexpr int kScoreWG = 4;                              // reducer warpgroups == TMEM buffers of 128 columns
+constexpr int kScoreWG = 2;                              // reducer warpgroups == TMEM buffers of 128 columns
 constexpr int kScoreThreads = 128 * kScoreWG + 64;       // + warp 4*WG: MMA + TMEM owner, warp 4*WG+1: TMA
-constexpr int kQStages = 3;
+constexpr int kQStages = 2;
 
 template <int D>
 struct ScoreSmem {
@@ -350,7 +350,7 @@ enum { C_KFULL = 0, C_QFULL = 1, C_QEMPTY = C_QFULL + kQStages, C_SFULL = C_QEMP
        C_SFREE = C_SFULL + kScoreWG, C_COUNT = C_SFREE + kScoreWG };
 
 template <int D>
-__global__ void __launch_bounds__(kScoreThreads, 1)
+__global__ void __launch_bounds__(kScoreThreads, 2)
 score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   using L = ScoreSmem<D>;
   constexpr int kMmaWarp = 4 * kScoreWG, kTmaWarp = 4 * kScoreWG + 1;
