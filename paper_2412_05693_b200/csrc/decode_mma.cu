@@ -117,8 +117,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
       qf[r][0] = w.x; qf[r][1] = w.y; qf[r][2] = w.z; qf[r][3] = w.w;
     }
   }
-  __syncthreads();
-
   const float sc2 = a.scale * kLog2e;
   const int n_iter = (n1 + kRowsPerIter - 1) / kRowsPerIter;   // same trip count for every thread
 
@@ -143,7 +141,12 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
   };
   {
     uint4 x[QR], y[QR];
-    load_k(0, x, y);
+    // the first tile of K does not contain the row appended above unless the cache is still tiny, so its loads
+    // are issued before the barrier that publishes that row
+    const bool early = c.n_old >= kRowsPerIter;
+    if (early) load_k(0, x, y);
+    __syncthreads();
+    if (!early) load_k(0, x, y);
     for (int it = 0; it < n_iter; ++it) {
       const int j0 = it * kRowsPerIter + warp * 16 + gid, j1 = j0 + 8;
       uint4 xn[QR], yn[QR];
@@ -181,8 +184,10 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
   }
   __syncthreads();
 
-  // ---- softmax over the n1 rows; the G heads are reduced side by side (independent shuffle chains)
-  float inv[G];
+  // ---- softmax statistics over the n1 rows with one barrier: every thread folds its own logits into a
+  // (maximum, sum of exp2 relative to that maximum) pair per head, pairs are merged across the warp by shuffles
+  // and across warps through shared memory in a fixed order.
+  float inv[G], mfin[G];
   {
     float m[G], t[G];
 #pragma unroll
@@ -191,41 +196,39 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
 #pragma unroll
       for (int h = 0; h < G; ++h) m[h] = fmaxf(m[h], s.p[h * n1t + j]);
 #pragma unroll
+    for (int h = 0; h < G; ++h) t[h] = 0.f;
+    for (int j = tid; j < n1; j += kThreads)
+#pragma unroll
+      for (int h = 0; h < G; ++h) t[h] += ex2f(s.p[h * n1t + j] - m[h]);   // ex2(-inf) = 0 when a thread has no row
+#pragma unroll
     for (int off = 16; off > 0; off >>= 1)
 #pragma unroll
-      for (int h = 0; h < G; ++h) m[h] = fmaxf(m[h], __shfl_xor_sync(0xffffffffu, m[h], off));
+      for (int h = 0; h < G; ++h) {
+        const float mo = __shfl_xor_sync(0xffffffffu, m[h], off), to = __shfl_xor_sync(0xffffffffu, t[h], off);
+        const float mn = fmaxf(m[h], mo);
+        // a side that has seen no row carries (-inf, 0): its term must not produce inf - inf
+        const float a0 = (m[h] == -INFINITY) ? 0.f : t[h] * ex2f(m[h] - mn);
+        const float a1 = (mo == -INFINITY) ? 0.f : to * ex2f(mo - mn);
+        // both lanes of a pair must add in the same order to stay bit-identical
+        t[h] = (lane & off) ? (a1 + a0) : (a0 + a1);
+        m[h] = mn;
+      }
     if (lane == 0)
 #pragma unroll
-      for (int h = 0; h < G; ++h) s.wred[h * kWarps + warp] = m[h];
+      for (int h = 0; h < G; ++h) { s.wred[h * kWarps + warp] = m[h]; s.wred[(G + h) * kWarps + warp] = t[h]; }
     __syncthreads();
 #pragma unroll
     for (int h = 0; h < G; ++h) {
       float mm = -INFINITY;
 #pragma unroll
       for (int w = 0; w < kWarps; ++w) mm = fmaxf(mm, s.wred[h * kWarps + w]);
-      m[h] = mm;
-      t[h] = 0.f;
-    }
-    for (int j = tid; j < n1; j += kThreads)
-#pragma unroll
-      for (int h = 0; h < G; ++h) {
-        const float e = ex2f(s.p[h * n1t + j] - m[h]);
-        s.p[h * n1t + j] = e;
-        t[h] += e;
-      }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1)
-#pragma unroll
-      for (int h = 0; h < G; ++h) t[h] += __shfl_xor_sync(0xffffffffu, t[h], off);
-    if (lane == 0)
-#pragma unroll
-      for (int h = 0; h < G; ++h) s.wred[(G + h) * kWarps + warp] = t[h];
-    __syncthreads();
-#pragma unroll
-    for (int h = 0; h < G; ++h) {
       float tt = 0.f;
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) tt += s.wred[(G + h) * kWarps + w];  // fixed order
+      for (int w = 0; w < kWarps; ++w) {   // fixed order
+        const float mw = s.wred[h * kWarps + w];
+        tt += (mw == -INFINITY) ? 0.f : s.wred[(G + h) * kWarps + w] * ex2f(mw - mm);
+      }
+      mfin[h] = mm;
       inv[h] = 1.f / tt;
     }
   }
@@ -242,7 +245,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
     float add = 0.f;
 #pragma unroll
     for (int h = 0; h < G; ++h) {
-      const float p = s.p[h * n1t + j] * inv[h];
+      const float p = ex2f(s.p[h * n1t + j] - mfin[h]) * inv[h];
       s.p[h * n1t + j] = p;
       add += p;
     }
