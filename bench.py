@@ -26,9 +26,8 @@ if ROOT not in sys.path:
 
 METRIC = "P&D evicting-attention tokens/s at max batch; % of TC (prefill) / HBM (decode) peak"
 UNIT = "tokens/s"
-# DRAM bytes per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
-# capture, see profiles/); None until a capture of the current kernel exists.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": {"attn_fwd": 91.9e6, "decode": None}}   # per launch, see profiles/
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the same command).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": {"attn_fwd": 91.9e6, "decode": 34.3e6}}   # profiles/attn_fwd_tc_cfg2_traffic.md
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 

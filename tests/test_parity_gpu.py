@@ -62,6 +62,42 @@ def test_cfg5_large_candidate_sets(B, K):
     run_lockstep(wl, [(1, 17)], check_rows_every=4)
 
 
+def test_cfg5_full_length_prompt():
+    # the largest candidate set of the table (2048 cached + 2048 new) at the full prompt length
+    wl = WORKLOADS["cfg5"].with_(b=2, B=2048, K=2048, steps=2)
+    run_lockstep(wl, [(0, 5)], check_rows_every=4)
+
+
+def test_cfg4_all_32_layers_share_one_handle():
+    wl = WORKLOADS["cfg4"].with_(b=2, s=1024, steps=2)
+    for layer in (0, 17, 31):
+        run_lockstep(wl, [(0, 0), (1, 7)], layer=layer, check_rows_every=2)
+
+
+def random_workloads(n, seed=2024):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        g = int(rng.choice([1, 2, 4, 8]))
+        hkv = int(rng.integers(1, 4))
+        d = int(rng.choice([64, 128]))
+        dtype = str(rng.choice(["bf16", "f32"]))
+        B = int(rng.integers(1, 200))
+        K = int(rng.integers(1, 300))
+        s = int(rng.integers(1, 700))
+        out.append(Workload(f"rand{i}_{dtype}_g{g}_d{d}_B{B}_K{K}_s{s}", b=int(rng.integers(1, 4)), Hq=g * hkv, Hkv=hkv,
+                            d=d, dtype=dtype, s=s, B=B, K=K, steps=int(rng.integers(0, 12)), seed=1000 + i,
+                            heavy_count=int(rng.integers(1, 9)), p_dec=int(rng.choice([1, 1, 3, 16]))))
+    return out
+
+
+@pytest.mark.parametrize("wl", random_workloads(10), ids=lambda w: w.name)
+def test_random_shapes(wl):
+    units = [(int(s), int(h)) for s in range(wl.b) for h in range(wl.Hkv)][:4]
+    st = run_lockstep(wl, units, check_rows_every=2)
+    assert st["calls"] == len(schedule(wl))
+
+
 # ------------------------------------------------------------------ shapes, tails and degenerate cases
 @pytest.mark.parametrize("wl", [
     tiny("ragged_f32"),                                               # I = 48, tail of 8, g = 2
