@@ -152,13 +152,16 @@ bm_status_t bm_prefill_block_static(bm_cache_t* cache, int32_t layer, int32_t sa
 /* ---- the same two passes fed from HOST memory (end-to-end use without device-side producers) ----
  * q/k/v/out are HOST pointers (pinned memory makes the copies asynchronous); `staging` is a DEVICE
  * buffer of at least bm_staging_bytes(cfg, nsamples, I) bytes.  The call copies q, k, v to the device,
- * runs the pass and copies out back to `out`; it does not synchronise.  The pass and the output copy are
- * ordered on cuda_stream (synchronising it makes `out` valid).  The input copies run on a stream owned by
- * the handle and start at call time, independent of cuda_stream's position, so q/k/v must hold their final
- * contents when the call is made and until cuda_stream has passed the call.  Passing two staging buffers
- * alternately lets the input copy of one call overlap the compute and output copy of the previous one; a
- * staging buffer is reused only after the earlier call that used it has finished (tracked by the handle).
- * While cuda_stream is being captured into a CUDA graph everything stays on cuda_stream. */
+ * runs the pass and copies out back to `out`; it does not synchronise.  The three stages run on streams
+ * owned by the handle, so that the input copy, the pass and the output copy of consecutive calls overlap;
+ * cuda_stream is made to wait for the call's output copy (synchronising cuda_stream makes `out` valid,
+ * and later work on cuda_stream sees the updated cache).  The pipeline is ordered after cuda_stream's
+ * position only where it has to be: at the first host-fed call and after any device-fed call on this
+ * handle.  The input copies start at call time, so q/k/v must hold their final contents when the call
+ * is made and until cuda_stream has passed the call.  Passing two staging buffers alternately keeps two
+ * calls in flight; a staging buffer is reused only after the earlier call that used it has finished
+ * (tracked by the handle).  While cuda_stream is being captured into a CUDA graph everything stays on
+ * cuda_stream. */
 bm_status_t bm_staging_bytes(const bm_config_t* cfg /*HOST*/, int32_t nsamples, int32_t I, size_t* bytes);
 bm_status_t bm_prefill_block_host(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples,
                                   const void* q /*HOST*/, const void* k /*HOST*/, const void* v /*HOST*/,

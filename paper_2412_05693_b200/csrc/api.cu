@@ -97,12 +97,18 @@ struct bm_cache {
   float* ws_lse;
   float* ws_new_sum;
   std::vector<int32_t> n, curr_id;  // [L * b] host mirror
-  // host-fed calls: inputs are copied on an internal stream so that the copy of one call overlaps the
-  // compute and the output copy of the previous one; two staging buffers can be in flight
-  cudaStream_t in_stream = nullptr;
-  struct Slot { void* staging = nullptr; cudaEvent_t in_done = nullptr; cudaEvent_t call_done = nullptr; };
+  // host-fed calls run as a three-stage pipeline on streams owned by the handle -- input copies, the pass,
+  // the output copy -- so that the three stages of consecutive calls overlap (PCIe is full duplex); the
+  // caller's stream only waits for each call's output copy.  Two staging buffers can be in flight.
+  cudaStream_t in_stream = nullptr, work_stream = nullptr, out_stream = nullptr;
+  cudaEvent_t entry_ev = nullptr;
+  struct Slot {
+    void* staging = nullptr;
+    cudaEvent_t in_done = nullptr, pass_done = nullptr, call_done = nullptr;
+  };
   Slot slots[2];
   int next_slot = 0;
+  long dev_calls = 0, dev_calls_seen = -1;  // device-fed calls made / already ordered before the pipeline
 };
 
 namespace {
@@ -226,12 +232,12 @@ bm_status_t bm_cache_destroy(bm_cache_t* cache) {
   if (cache == nullptr) return BM_ERR_INVALID;
   if (cache->in_stream != nullptr) {
     cudaSetDevice(cache->cfg.device);
-    cudaStreamSynchronize(cache->in_stream);
-    for (auto& sl : cache->slots) {
-      if (sl.in_done) cudaEventDestroy(sl.in_done);
-      if (sl.call_done) cudaEventDestroy(sl.call_done);
-    }
-    cudaStreamDestroy(cache->in_stream);
+    for (cudaStream_t st : {cache->in_stream, cache->work_stream, cache->out_stream})
+      if (st != nullptr) { cudaStreamSynchronize(st); cudaStreamDestroy(st); }
+    for (auto& sl : cache->slots)
+      for (cudaEvent_t ev : {sl.in_done, sl.pass_done, sl.call_done})
+        if (ev) cudaEventDestroy(ev);
+    if (cache->entry_ev) cudaEventDestroy(cache->entry_ev);
   }
   delete cache;
   return BM_OK;
@@ -248,6 +254,7 @@ bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int3
   int n_old = 0, curr = 0;
   bm_status_t s = check_range(c, layer, sample0, nsamples, &n_old, &curr);
   if (s != BM_OK) return s;
+  ++c->dev_calls;  // a later host-fed call orders its pipeline after this one
   if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) return BM_ERR_INVALID;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BM_ERR_INVALID;
   if (I < 1 || I > c->cfg.block_max) return BM_ERR_INVALID;
@@ -295,6 +302,7 @@ bm_status_t bm_decode_step(bm_cache_t* c, int32_t layer, int32_t sample0, int32_
   int n_old = 0, curr = 0;
   bm_status_t s = check_range(c, layer, sample0, nsamples, &n_old, &curr);
   if (s != BM_OK) return s;
+  ++c->dev_calls;  // a later host-fed call orders its pipeline after this one
   if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) return BM_ERR_INVALID;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BM_ERR_INVALID;
   const int n1 = n_old + 1;
@@ -324,6 +332,7 @@ bm_status_t bm_evict(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsam
   int n_old = 0, curr = 0;
   bm_status_t s = check_range(c, layer, sample0, nsamples, &n_old, &curr);
   if (s != BM_OK) return s;
+  ++c->dev_calls;  // a later host-fed call orders its pipeline after this one
   if (target < 0) return BM_ERR_INVALID;
   if (n_old <= target) return BM_OK;
   if (target == 0) { set_mirror(c, layer, sample0, nsamples, 0, curr); return BM_OK; }
@@ -387,20 +396,32 @@ static bm_status_t host_pass(bm_cache_t* c, int layer, int sample0, int nsamples
   cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
   cudaStreamIsCapturing(st, &cap);
   bm_cache::Slot* slot = nullptr;
-  cudaStream_t in = st;
+  cudaStream_t in = st, work = st, outs = st;
   if (cap == cudaStreamCaptureStatusNone) {
     if (c->in_stream == nullptr) {
-      if (cudaStreamCreateWithFlags(&c->in_stream, cudaStreamNonBlocking) != cudaSuccess) return BM_ERR_CUDA;
-      for (auto& sl : c->slots) {
-        if (cudaEventCreateWithFlags(&sl.in_done, cudaEventDisableTiming) != cudaSuccess ||
-            cudaEventCreateWithFlags(&sl.call_done, cudaEventDisableTiming) != cudaSuccess)
-          return BM_ERR_CUDA;
-      }
+      bool ok = cudaStreamCreateWithFlags(&c->in_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                cudaStreamCreateWithFlags(&c->work_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                cudaEventCreateWithFlags(&c->entry_ev, cudaEventDisableTiming) == cudaSuccess;
+      for (auto& sl : c->slots)
+        ok = ok && cudaEventCreateWithFlags(&sl.in_done, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&sl.pass_done, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&sl.call_done, cudaEventDisableTiming) == cudaSuccess;
+      if (!ok) return BM_ERR_CUDA;
     }
     for (auto& sl : c->slots)
       if (sl.staging == staging) slot = &sl;
     if (slot == nullptr) { slot = &c->slots[c->next_slot]; c->next_slot ^= 1; }
     in = c->in_stream;
+    work = c->work_stream;
+    outs = c->out_stream;
+    // Device-fed calls (and the creation of the cache) since the last host-fed one are ordered before the
+    // pipeline through cuda_stream.  Consecutive host-fed calls skip this, or each pass would wait for the
+    // previous call's output copy, which cuda_stream has been made to wait for.
+    if (c->dev_calls_seen != c->dev_calls) {
+      if (cudaEventRecord(c->entry_ev, st) != cudaSuccess || cudaStreamWaitEvent(work, c->entry_ev, 0) != cudaSuccess)
+        return BM_ERR_CUDA;
+    }
     // the staging buffer is free again once the previous call that used this slot has finished with it
     if (slot->staging != nullptr && cudaStreamWaitEvent(in, slot->call_done, 0) != cudaSuccess) return BM_ERR_CUDA;
     slot->staging = staging;
@@ -410,14 +431,22 @@ static bm_status_t host_pass(bm_cache_t* c, int layer, int sample0, int nsamples
   if (cudaMemcpyAsync(sp + ov, v, kb, cudaMemcpyHostToDevice, in) != cudaSuccess) return BM_ERR_CUDA;
   if (slot != nullptr) {
     if (cudaEventRecord(slot->in_done, in) != cudaSuccess) return BM_ERR_CUDA;
-    if (cudaStreamWaitEvent(st, slot->in_done, 0) != cudaSuccess) return BM_ERR_CUDA;
+    if (cudaStreamWaitEvent(work, slot->in_done, 0) != cudaSuccess) return BM_ERR_CUDA;
   }
-  s = decode ? bm_decode_step(c, layer, sample0, nsamples, sp + oq, sp + ok, sp + ov, sp + oo, evict_to, cuda_stream)
+  s = decode ? bm_decode_step(c, layer, sample0, nsamples, sp + oq, sp + ok, sp + ov, sp + oo, evict_to, work)
              : bm_prefill_block(c, layer, sample0, nsamples, sp + oq, sp + ok, sp + ov, I, pos0, sp + oo, evict_to,
-                                cuda_stream);
+                                work);
   if (s != BM_OK) return s;
-  if (cudaMemcpyAsync(out, sp + oo, qb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return BM_ERR_CUDA;
-  if (slot != nullptr && cudaEventRecord(slot->call_done, st) != cudaSuccess) return BM_ERR_CUDA;
+  if (slot != nullptr) {
+    c->dev_calls_seen = c->dev_calls;
+    if (cudaEventRecord(slot->pass_done, work) != cudaSuccess) return BM_ERR_CUDA;
+    if (cudaStreamWaitEvent(outs, slot->pass_done, 0) != cudaSuccess) return BM_ERR_CUDA;
+  }
+  if (cudaMemcpyAsync(out, sp + oo, qb, cudaMemcpyDeviceToHost, outs) != cudaSuccess) return BM_ERR_CUDA;
+  if (slot != nullptr) {
+    if (cudaEventRecord(slot->call_done, outs) != cudaSuccess) return BM_ERR_CUDA;
+    if (cudaStreamWaitEvent(st, slot->call_done, 0) != cudaSuccess) return BM_ERR_CUDA;
+  }
   return BM_OK;
 }
 
@@ -494,6 +523,7 @@ bm_status_t bm_cache_import(bm_cache_t* c, int32_t layer, int32_t sample, int32_
   if (kv_ids == nullptr || sum_weights == nullptr || k_rows == nullptr || v_rows == nullptr) return BM_ERR_INVALID;
   if (n != c->n[(size_t)layer * c->cfg.batch + sample]) return BM_ERR_STATE;
   if ((s = set_device(c)) != BM_OK) return s;
+  ++c->dev_calls;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t rb = (size_t)c->cfg.head_dim * c->esz;
   bool ok = true;

@@ -192,20 +192,24 @@ def run_free(wl, host=False, micro=None):
     cfg = make_config(wl)
     cache = bm.BatchMaxCache(cfg)
     inp = Inputs(wl, "cuda")
-    outs = []
+    outs, keep = [], []
     for kind, pos0, I, ev in schedule(wl):
         q, k, v = inp.block(0, pos0, I)
         if kind == "decode":
             q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
-        if host:
+        if host and not (host == "mixed" and len(outs) % 2 == 1):
             qh, kh, vh = (t.cpu().pin_memory() for t in (q, k, v))
             oh = torch.empty_like(qh).pin_memory()
             if kind == "prefill":
                 cache.prefill_block_host(qh, kh, vh, pos0, oh, evict_to=ev)
             else:
                 cache.decode_step_host(qh, kh, vh, oh, evict_to=ev)
-            torch.cuda.synchronize()
-            outs.append(oh.clone())
+            if host is True:
+                torch.cuda.synchronize()
+                outs.append(oh.clone())
+            else:               # calls stay in flight; only the caller's stream is synchronised at the end
+                outs.append(oh)
+                keep.append((qh, kh, vh))
         elif micro and kind == "prefill":
             o = torch.empty_like(q)
             for s0 in range(0, wl.b, micro):
@@ -221,7 +225,9 @@ def run_free(wl, host=False, micro=None):
         else:
             o = cache.prefill_block(q, k, v, pos0, evict_to=ev) if kind == "prefill" else \
                 cache.decode_step(q, k, v, evict_to=ev)
-            outs.append(o.cpu())
+            outs.append(o if host else o.cpu())
+    torch.cuda.current_stream().synchronize()
+    outs = [o.cpu().clone() for o in outs]
     state = [cache.export(0, s, h, rows=True) for s in range(wl.b) for h in range(wl.Hkv)]
     cache.close()
     return outs, state
@@ -241,6 +247,8 @@ def test_bitwise_reproducible_and_variants_agree(dtype, d):
     base = run_free(wl)
     assert_same_run(base, run_free(wl))                 # run-to-run determinism (no float atomics)
     assert_same_run(base, run_free(wl, host=True))      # host-fed entry points
+    assert_same_run(base, run_free(wl, host="pipelined"))   # ... with every call left in flight
+    assert_same_run(base, run_free(wl, host="mixed"))       # ... alternating with device-fed calls, no syncs
     assert_same_run(base, run_free(wl, micro=1))        # sample ranges: micro-batched calls
 
 
