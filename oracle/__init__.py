@@ -10,4 +10,5 @@ from .batchmax_oracle import (  # noqa: F401
     run_north_star,
     run_algorithm1,
     run_decode_only,
+    run_extreme_decoding,
 )

@@ -26,6 +26,11 @@ Readings of points the paper leaves open (each is a convention of this build):
   * survivors keep their sum_weights (the vector is "variable-sized": entries
     leave with their pairs and nothing is reset).
 
+The extreme decoding-only comparison of Algorithm 3 (keep only the most recent
+pair) is here as well, :meth:`UnitCache.keep_most_recent` and
+:func:`run_extreme_decoding`, because the library's timed comparison arm is
+checked against it.
+
 Parity unpinned (conventions, not derivable from the paper): the GQA sum, the
 tie direction and the denominator reading above.  Everything else is pinned by
 tests/test_oracle_pins.py.
@@ -160,6 +165,22 @@ class UnitCache:
         return snap
 
 
+    # ------------------------------------------------------------------ Algorithm 3's rule
+    def keep_most_recent(self, keep: int = 1):
+        """Remove all but the ``keep`` most recent pairs (the rule of the extreme decoding-only
+        comparison, Algorithm 3, where keep = 1).  Survivors keep their sum_weights."""
+        n = len(self)
+        keep = int(keep)
+        if keep >= n:
+            return
+        first = n - keep
+        self.evicted_mass += float(self.sum_weights[:first].sum())
+        self.kv_ids = self.kv_ids[first:]
+        self.k = self.k[first:]
+        self.v = self.v[first:]
+        self.sum_weights = self.sum_weights[first:]
+
+
 # ---------------------------------------------------------------------- plain definition
 def dense_causal_attention(q, k, v, scale: float | None = None):
     """Full-KV-cache attention (the no-eviction limit, "FKV" in Sec. 4), written out from the
@@ -258,3 +279,29 @@ def run_decode_only(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec:
         outs.append(unit.decode_step(q[s + t], k[s + t], v[s + t], kv_max if full else -1)[None])
         trace.append(_trace_entry(unit))
     return np.concatenate(outs, axis=0), trace, unit
+
+
+def run_extreme_decoding(q, k, v, s: int, kv_bar: int, max_gen: int, block: int | None = None,
+                         scale: float | None = None):
+    """Algorithm 3 (extreme decoding-only eviction): the whole prompt is processed with a full
+    cache (in blocks of ``block`` positions when given; the split changes nothing but rounding),
+    all but the most recent pair are removed, and for t = 1..max_gen-1 the token at position
+    s + t - 1 is processed, after which a cache that holds kv_bar pairs is cut back to its most
+    recent pair."""
+    q = np.asarray(q, dtype=np.float64)
+    unit = UnitCache(q.shape[2], q.shape[1], scale)
+    outs, sizes = [], []
+    block = s if block is None else block
+    pos = 0
+    while pos < s:
+        I = min(block, s - pos)
+        outs.append(unit.process_block(q[pos:pos + I], k[pos:pos + I], v[pos:pos + I], pos))
+        pos += I
+    unit.keep_most_recent(1)
+    for t in range(1, max_gen):
+        pos = s + t - 1
+        outs.append(unit.decode_step(q[pos], k[pos], v[pos])[None])
+        sizes.append(len(unit))
+        if len(unit) == kv_bar:
+            unit.keep_most_recent(1)
+    return np.concatenate(outs, axis=0), unit, sizes

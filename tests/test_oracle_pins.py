@@ -10,7 +10,8 @@ import numpy as np
 import pytest
 import torch
 
-from oracle import UnitCache, dense_causal_attention, run_algorithm1, run_decode_only, run_north_star
+from oracle import (UnitCache, dense_causal_attention, run_algorithm1, run_decode_only, run_extreme_decoding,
+                    run_north_star)
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "sec3_2_closed_forms.txt")
 
@@ -444,3 +445,54 @@ def test_kept_override_for_lockstep():
     snap = u.evict(5, kept_ids=[0, 2, 4, 6, 8])
     assert list(u.kv_ids) == [0, 2, 4, 6, 8]
     assert len(snap["kept_ids"]) == 5 and snap["cand_ids"].shape[0] == 10
+
+
+# ---------------------------------------------------------------- Algorithm 3 (extreme decoding-only eviction)
+def windowed_attention(q, k, v, visible, scale):
+    """Row i attends to the positions visible(i); written straight from the softmax definition."""
+    out = np.zeros((q.shape[0], q.shape[1], v.shape[1]))
+    for i in range(q.shape[0]):
+        js = visible(i)
+        for h in range(q.shape[1]):
+            logits = np.array([scale * float(q[i, h] @ k[j]) for j in js])
+            w = np.exp(logits - logits.max())
+            w /= w.sum()
+            out[i, h] = sum(wj * v[j] for wj, j in zip(w, js))
+    return out
+
+
+@pytest.mark.parametrize("kv_bar,block", [(2, None), (2, 5), (5, None), (65, 7)])
+def test_extreme_decoding_is_prompt_dense_then_window_since_last_cut(kv_bar, block):
+    # Algorithm 3: the prompt sees everything; afterwards the cache is the pair kept at the last cut plus
+    # what was generated since, so with a limit of 2 every decode query sees its predecessor and itself.
+    s, g, d, max_gen = 23, 2, 8, 80
+    q, k, v = rand_qkv(31, s + max_gen, g, d)
+    out, unit, sizes = run_extreme_decoding(q, k, v, s, kv_bar, max_gen, block=block)
+    scale = 1.0 / math.sqrt(d)
+
+    def visible(i):
+        if i < s:
+            return list(range(i + 1))
+        t = i - s                               # decode forwards since the prompt
+        anchor = s - 1 + (t // (kv_bar - 1)) * (kv_bar - 1)   # pair kept at the most recent cut
+        return list(range(anchor, i + 1))
+
+    n_rows = s + max_gen - 1
+    np.testing.assert_allclose(out, windowed_attention(q[:n_rows], k, v, visible, scale), atol=1e-12)
+    assert max(sizes) == kv_bar and min(sizes) == 2
+    assert len(unit) == (1 if (max_gen - 1) % (kv_bar - 1) == 0 else 1 + (max_gen - 1) % (kv_bar - 1))
+    # mass conservation also holds under this rule
+    assert unit.sum_weights.sum() + unit.evicted_mass == pytest.approx(g * n_rows, rel=1e-12)
+
+
+def test_keep_most_recent_keeps_ids_and_sums_of_the_tail():
+    u = UnitCache(4, 1)
+    q, k, v = rand_qkv(5, 9, 1, 4)
+    u.process_block(q, k, v, 0)
+    before = (u.kv_ids.copy(), u.sum_weights.copy(), u.k.copy(), u.v.copy())
+    u.keep_most_recent(3)
+    assert list(u.kv_ids) == [6, 7, 8]
+    for a, b in zip(before, (u.kv_ids, u.sum_weights, u.k, u.v)):
+        assert np.array_equal(a[6:], b)
+    u.keep_most_recent(5)                       # nothing to remove
+    assert len(u) == 3
