@@ -130,6 +130,15 @@ bm_status_t bm_decode_step(bm_cache_t* cache, int32_t layer, int32_t sample0, in
 bm_status_t bm_evict(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples, int32_t target,
                      void* cuda_stream);
 
+/* ---- the rule of the extreme decoding-only comparison (Algorithm 3: "remove all but the most recent
+ * KV pair") ----
+ * Keep the `keep` most recent pairs of every cache of the range, moved to the front with their
+ * sum_weights and kv_ids; n becomes keep.  No-op when n <= keep.  It exists so that the comparison arm
+ * of the paper's experiments (Sec. 5, ED) runs on the same kernels and memory model as the method itself.
+ * Errors as bm_evict. */
+bm_status_t bm_keep_most_recent(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples,
+                                int32_t keep, void* cuda_stream);
+
 /* ---- bm_prefill_block for callers that cannot provide scratch (the paper has no counterpart) ----
  * Identical to bm_prefill_block in arguments, result and errors, but the per-call scratch (log-sum-exp of
  * the query rows, column sums of the new pairs) is taken from a fixed 5 MiB array that is part of the

@@ -47,6 +47,7 @@ SIGNATURES = {
     "bm_prefill_block_static": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _vp, _i32, _vp]),
     "bm_decode_step": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp]),
     "bm_evict": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp]),
+    "bm_keep_most_recent": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp]),
     "bm_staging_bytes": (_i32, [_cfgp, _i32, _i32, C.POINTER(_sz)]),
     "bm_prefill_block_host": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
     "bm_decode_step_host": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp, _sz, _vp]),
@@ -251,6 +252,12 @@ class BatchMaxCache:
     def evict(self, target: int, layer: int = 0, sample0: int = 0, nsamples: int | None = None, stream=None):
         ns = self.cfg.batch - sample0 if nsamples is None else nsamples
         _check(lib().bm_evict(self.h, layer, sample0, ns, target, _stream(stream)), "bm_evict")
+
+    def keep_most_recent(self, keep: int = 1, layer: int = 0, sample0: int = 0, nsamples: int | None = None,
+                         stream=None):
+        """Algorithm 3's rule: all but the `keep` most recent pairs leave the cache."""
+        ns = self.cfg.batch - sample0 if nsamples is None else nsamples
+        _check(lib().bm_keep_most_recent(self.h, layer, sample0, ns, keep, _stream(stream)), "bm_keep_most_recent")
 
     # -- host-fed variants ---------------------------------------------------------------------------
     def _stage(self, ns, I):

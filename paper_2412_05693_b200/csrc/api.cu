@@ -327,8 +327,8 @@ bm_status_t bm_decode_step(bm_cache_t* c, int32_t layer, int32_t sample0, int32_
   return BM_OK;
 }
 
-bm_status_t bm_evict(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, int32_t target,
-                     void* cuda_stream) {
+static bm_status_t evict_cached(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, int32_t target,
+                                bool recent, void* cuda_stream) {
   int n_old = 0, curr = 0;
   bm_status_t s = check_range(c, layer, sample0, nsamples, &n_old, &curr);
   if (s != BM_OK) return s;
@@ -341,10 +341,20 @@ bm_status_t bm_evict(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsam
   CacheView view = make_view(c, layer, sample0, nsamples, n_old);
   EvictArgs e;
   e.blk_k = nullptr; e.blk_v = nullptr; e.new_sum = nullptr;
-  e.I = 0; e.pos0 = 0; e.curr_id = curr; e.target = target;
+  e.I = 0; e.pos0 = 0; e.curr_id = curr; e.target = target; e.recent = recent ? 1 : 0;
   if ((s = run_evict(c, view, e, static_cast<cudaStream_t>(cuda_stream))) != BM_OK) return s;
   set_mirror(c, layer, sample0, nsamples, target, curr);
   return BM_OK;
+}
+
+bm_status_t bm_evict(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, int32_t target,
+                     void* cuda_stream) {
+  return evict_cached(c, layer, sample0, nsamples, target, false, cuda_stream);
+}
+
+bm_status_t bm_keep_most_recent(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, int32_t keep,
+                                void* cuda_stream) {
+  return evict_cached(c, layer, sample0, nsamples, keep, true, cuda_stream);
 }
 
 // ---- host-fed variants ---------------------------------------------------------------------------

@@ -41,6 +41,7 @@ struct EvictArgs {
   int32_t pos0;
   int32_t curr_id;       // last processed position
   int32_t target;        // pairs to keep (<= n_old + I)
+  int32_t recent = 0;    // 1: keep the `target` most recent candidates instead of ranking by ave_weights
 };
 
 // Launchers (host).  All enqueue on `st` and return the CUDA error of the launch.

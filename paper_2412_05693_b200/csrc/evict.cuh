@@ -2,6 +2,8 @@
 //   ave_weights = sum_weights / (g * (curr_id + 1 - kv_ids)),
 // keep the `target` candidates ranking first under (ave_weights descending, kv_ids ascending),
 // then compact rows, sum_weights and kv_ids to the front of the cache in ascending kv_ids order.
+// (EvictArgs::recent selects the rule of the extreme decoding-only comparison instead, Algorithm 3:
+// the `target` most recent candidates stay.)
 // Candidates are the n_old cached pairs followed by I new pairs that still live in the caller's
 // block buffers; both lists are ascending in kv_ids, so candidate index order is kv_ids order.
 #pragma once
@@ -76,6 +78,9 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
 
   if (target >= n_c) {
     for (int r = tid; r < n_c; r += NT) s.src[r] = r;
+    __syncthreads();
+  } else if (e.recent) {  // Algorithm 3's rule: the most recent pairs stay, whatever their weights
+    for (int r = tid; r < target; r += NT) s.src[r] = n_c - target + r;
     __syncthreads();
   } else {
     // ---- radix select: bit pattern `thr` of the target-th largest ave, and how many equal to it to keep

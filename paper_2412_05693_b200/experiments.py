@@ -4,6 +4,7 @@
     python -m paper_2412_05693_b200.experiments --run cfg3_ratio    # P&D vs decode-only compression, same arena
     python -m paper_2412_05693_b200.experiments --run cfg4          # 32 layers, batch that fills 120 GiB
     python -m paper_2412_05693_b200.experiments --run cfg5          # the six (block, kv_max) combinations
+    python -m paper_2412_05693_b200.experiments --run sec5          # Sec. 5's arms: BM (Algorithm 1) vs ED vs FKV
 
 Batches this large cannot keep their prompts resident (one block of cfg3 at b = 10072 is 63 GB of Q/K/V), so
 inputs are drawn on the fly per (layer, block, range of samples) from the seeded generator and every library
@@ -40,11 +41,80 @@ def peaks():
 DECODE_MICRO = 2048   # samples per decode call (decode inputs are tiny, so ranges can be much wider than in prefill)
 
 
-def make_cfg(wl: Workload, batch: int, arm: str, micro: int, device: int = 0) -> Config:
-    growth = max(1, wl.p_dec) if arm == "pd" else wl.s + max(1, wl.p_dec) - wl.K
-    return Config(batch=batch, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.d, kv_max=wl.K, block_max=wl.B,
+ARMS = {
+    "pd": "Batch-Max in the build's cadence: evict to K after every block and (when full) decode step",
+    "do": "decoding-only compression (Sec. 1): whole prompt cached, one compression to K, then as pd",
+    "alg1": "Batch-Max exactly as Algorithm 1: limit kv_bar, p pairs removed before each block of p / when full",
+    "ed": "extreme decoding-only eviction (Algorithm 3): whole prompt cached, then only the newest pair kept",
+    "fkv": "full KV cache: nothing is ever removed",
+}
+
+
+def make_cfg(wl: Workload, batch: int, arm: str, micro: int, device: int = 0, kv_bar: int | None = None,
+             p: int = 64) -> Config:
+    """Cache geometry of an arm; cap = kv_max + growth is what the memory model charges per cache."""
+    block = wl.B
+    if arm == "pd":
+        kv_max, growth = wl.K, max(1, wl.p_dec)
+    elif arm == "do":
+        kv_max, growth = wl.K, wl.s + max(1, wl.p_dec) - wl.K
+    elif arm == "alg1":
+        kv_max, growth, block = kv_bar - p, p, max(p, min(wl.B, kv_bar))      # cap = kv_bar
+    elif arm == "ed":
+        kv_max, growth = wl.s, max(1, kv_bar - 1)                              # prompt, then <= kv_bar pairs
+    elif arm == "fkv":
+        kv_max, growth = wl.s, max(1, wl.steps)
+    else:
+        raise ValueError(arm)
+    return Config(batch=batch, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.d, kv_max=kv_max, block_max=block,
                   growth=growth, dtype=wl.dtype, n_layers=wl.L, device=device,
                   max_call_samples=max(micro, min(batch, DECODE_MICRO)))
+
+
+def arm_calls(wl: Workload, arm: str, kv_bar: int | None = None, p: int = 64):
+    """Calls of one layer as (kind, pos0, I, arg): kind in prefill / decode (arg = evict_to, -1 for none),
+    evict (arg = target), recent (arg = pairs kept)."""
+    calls, n = [], 0
+    if arm == "alg1":
+        # first min(s, kv_bar) tokens without eviction (any split gives the same result), then p out, <= p in
+        t1 = min(wl.s, kv_bar)
+        blk = max(p, min(wl.B, kv_bar))
+        for pos0 in range(0, t1, blk):
+            calls.append(("prefill", pos0, min(blk, t1 - pos0), -1))
+        n = t1
+        while t1 < wl.s:
+            calls.append(("evict", 0, 0, n - p))
+            I = min(p, wl.s - t1)
+            calls.append(("prefill", t1, I, -1))
+            n, t1 = n - p + I, t1 + I
+        for t in range(wl.steps):
+            if n == kv_bar:
+                calls.append(("evict", 0, 0, n - p))
+                n -= p
+            calls.append(("decode", wl.s + t, 1, -1))
+            n += 1
+        return calls
+    for pos0 in range(0, wl.s, wl.B):
+        calls.append(("prefill", pos0, min(wl.B, wl.s - pos0), wl.K if arm == "pd" else -1))
+    n = min(wl.s, wl.K) if arm == "pd" else wl.s
+    if arm == "do":
+        calls.append(("evict", 0, 0, wl.K))
+        n = min(n, wl.K)
+    if arm == "ed":
+        calls.append(("recent", 0, 0, 1))
+        n = 1
+    for t in range(wl.steps):
+        if arm in ("pd", "do"):
+            full = n + 1 >= wl.K + wl.p_dec
+            calls.append(("decode", wl.s + t, 1, wl.K if full else -1))
+            n = wl.K if full else n + 1
+        else:
+            calls.append(("decode", wl.s + t, 1, -1))
+            n += 1
+            if arm == "ed" and n == kv_bar:
+                calls.append(("recent", 0, 0, 1))
+                n = 1
+    return calls
 
 
 class Timer:
@@ -65,12 +135,11 @@ class Timer:
         return t
 
 
-def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=None, device: int = 0):
-    """One arm over the whole schedule.  arm 'pd': evict to K after every block and decode step (P&D);
-    arm 'do': cache the whole prompt, compress to K once after it, then decode with eviction (decode-only
-    compression, Sec. 1).  Returns a dict of timings and derived rates."""
+def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=None, device: int = 0,
+            kv_bar: int | None = None, p: int = 64):
+    """One arm (see ARMS) over the whole schedule.  Returns a dict of timings and derived rates."""
     wl = wl.with_(b=batch)
-    cfg = make_cfg(wl, batch, arm, micro, device)
+    cfg = make_cfg(wl, batch, arm, micro, device, kv_bar, p)
     dev = torch.device("cuda", device)
     need = arena_bytes(cfg)
     if arena is None:
@@ -81,52 +150,59 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
     t_pre, t_dec = Timer(), Timer()
     ms_pre = ms_dec = 0.0
     layers = range(wl.L) if layers is None else layers
-    out_blk = torch.empty(micro, wl.B, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
+    out_blk = torch.empty(micro, cfg.block_max, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
     micro_dec = max(micro, min(batch, DECODE_MICRO))
     out_dec = torch.empty(micro_dec, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
-    pairs = 0
+    calls = arm_calls(wl, arm, kv_bar, p)
+    pairs = dec_rows = 0
     for layer in layers:
-        n = 0
-        for pos0 in range(0, wl.s, wl.B):
-            I = min(wl.B, wl.s - pos0)
-            ev = wl.K if arm == "pd" else -1
-            for s0 in range(0, batch, micro):
-                ns = min(micro, batch - s0)
-                q, k, v = inp.block(layer, pos0, I, s0, ns)
-                t_pre(lambda: cache.prefill_block(q, k, v, pos0, out=out_blk[:ns, :I], evict_to=ev, layer=layer,
-                                                  sample0=s0))
-            pairs += I * n + I * (I + 1) // 2
-            n = min(n + I, wl.K) if arm == "pd" else n + I
-            ms_pre += t_pre.total_ms()
-        if arm == "do":
-            for s0 in range(0, batch, micro):
-                ns = min(micro, batch - s0)
-                t_pre(lambda: cache.evict(wl.K, layer=layer, sample0=s0, nsamples=ns))
-            n = min(n, wl.K)
-            ms_pre += t_pre.total_ms()
-        for t in range(wl.steps):
-            full = n + 1 >= wl.K + wl.p_dec
-            ev = wl.K if full else -1
-            for s0 in range(0, batch, micro_dec):
-                ns = min(micro_dec, batch - s0)
-                q, k, v = inp.block(layer, wl.s + t, 1, s0, ns)
-                q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
-                t_dec(lambda: cache.decode_step(q, k, v, out=out_dec[:ns], evict_to=ev, layer=layer, sample0=s0))
-            n = wl.K if full else n + 1
-            if (t & 15) == 15 or t == wl.steps - 1:
+        n, in_decode, pending = 0, False, 0
+        for kind, pos0, I, arg in calls:
+            in_decode = in_decode or kind == "decode"
+            timer = t_dec if in_decode else t_pre
+            if kind == "prefill":
+                for s0 in range(0, batch, micro):
+                    ns = min(micro, batch - s0)
+                    q, k, v = inp.block(layer, pos0, I, s0, ns)
+                    timer(lambda: cache.prefill_block(q, k, v, pos0, out=out_blk[:ns, :I], evict_to=arg, layer=layer,
+                                                      sample0=s0))
+                pairs += I * n + I * (I + 1) // 2
+                n = n + I if arg < 0 else min(n + I, arg)
+            elif kind == "decode":
+                for s0 in range(0, batch, micro_dec):
+                    ns = min(micro_dec, batch - s0)
+                    q, k, v = inp.block(layer, pos0, 1, s0, ns)
+                    q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
+                    timer(lambda: cache.decode_step(q, k, v, out=out_dec[:ns], evict_to=arg, layer=layer, sample0=s0))
+                dec_rows += n + 1
+                n = n + 1 if arg < 0 else min(n + 1, arg)
+            else:
+                rule = cache.evict if kind == "evict" else cache.keep_most_recent
+                step = micro_dec if in_decode else micro
+                for s0 in range(0, batch, step):
+                    ns = min(step, batch - s0)
+                    timer(lambda: rule(arg, layer=layer, sample0=s0, nsamples=ns))
+                n = min(n, arg)
+            pending += 1
+            if pending >= 16:
+                ms_pre += t_pre.total_ms()
                 ms_dec += t_dec.total_ms()
+                pending = 0
+        ms_pre += t_pre.total_ms()
+        ms_dec += t_dec.total_ms()
     assert cache.status() == 0
     n_layers = len(list(layers))
     n_end, cur = cache.length(layer=list(layers)[-1], sample=batch - 1)
+    assert n_end == n, "host mirror disagrees with the schedule's own count"
     cache.close()
     hbm, tf, src = peaks()
     e = wl.elem_bytes
     flops = 4.0 * wl.d * (pairs / n_layers) * batch * wl.Hq * n_layers
-    n1 = min(wl.K, wl.s) + 1
-    dec_bytes = batch * wl.Hkv * n_layers * wl.steps * (n1 * (2 * wl.d * e + 16) + 2 * wl.d * e + 2 * wl.g * wl.d * e)
+    dec_bytes = batch * wl.Hkv * n_layers * ((dec_rows / n_layers) * (2 * wl.d * e + 16)
+                                             + wl.steps * (2 * wl.d * e + 2 * wl.g * wl.d * e))
     res = {
         "workload": wl.name, "arm": arm, "batch": batch, "layers_run": n_layers, "micro_batch": micro,
-        "decode_micro_batch": micro_dec,
+        "decode_micro_batch": micro_dec, "cap": cfg.kv_max + cfg.growth,
         "arena_GiB": need / GiB, "final_n": n_end, "final_curr_id": cur,
         "prefill_ms": ms_pre, "decode_ms": ms_dec,
         "prefill_tok_s": batch * wl.s * n_layers / (ms_pre * 1e-3),
@@ -137,15 +213,20 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
         "decode_gbs": dec_bytes / (ms_dec * 1e-3) / 1e9 if ms_dec > 0 else None,
         "decode_frac_of_peak": dec_bytes / (ms_dec * 1e-3) / 1e9 / hbm if ms_dec > 0 else None,
         "peaks": {"hbm_gbs": hbm, "bf16_tflops_sustained": tf, "source": src},
-        "note": "prefill = all bm_prefill_block calls incl. score pass and eviction (whole call, not the forward kernel "
-                "alone); decode bytes exclude compaction moves; every call timed with its own CUDA events",
+        "note": "prefill = every call before the first decode step (attention, score pass, evictions; the whole call, "
+                "not the forward kernel alone); decode = every call from the first decode step on; decode bytes "
+                "exclude compaction moves; every call timed with its own CUDA events",
     }
+    if arm in ("alg1", "ed"):
+        res["kv_bar"] = kv_bar
+    if arm == "alg1":
+        res["p"] = p
     return res
 
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--run", required=True, choices=["cfg3_max", "cfg3_ratio", "cfg4", "cfg5"])
+    ap.add_argument("--run", required=True, choices=["cfg3_max", "cfg3_ratio", "cfg4", "cfg5", "sec5"])
     ap.add_argument("--budget-gib", type=float, default=None)
     ap.add_argument("--micro", type=int, default=256)
     ap.add_argument("--layers", type=int, default=None, help="run only the first N layers (cfg4)")
@@ -178,6 +259,20 @@ def main():
         layers = range(wl.L) if args.layers is None else range(args.layers)
         res = run_arm(wl, b, "pd", args.micro, arena=arena, layers=layers)
         print(json.dumps({"run": "cfg4", "budget_GiB": budget / GiB, "batch": b, "pd": res}))
+    elif args.run == "sec5":
+        # The procedure of Sec. 5 on one attention layer of the larger model's shape (40 heads of 128, prompt
+        # 3584, 512 tokens generated = 511 decode forwards): every arm runs at the largest batch whose caches
+        # fit the same budget.  Only cache memory is modelled, so the batch ratios are those of the caches alone.
+        wl = Workload("sec5", b=1, Hq=40, Hkv=40, d=128, dtype="bf16", s=3584, B=512, K=1024,
+                      steps=args.decode_steps if args.decode_steps is not None else 511, seed=5, heavy_count=36)
+        budget = int((args.budget_gib or 4.0) * GiB)
+        arena = torch.empty(budget, dtype=torch.uint8, device="cuda")
+        arms = [("alg1", 1024), ("alg1", 2048), ("ed", 2), ("ed", 65), ("fkv", None)]
+        for arm, kv_bar in arms:
+            b = max_batch(make_cfg(wl, 1, arm, args.micro, kv_bar=kv_bar), budget)
+            res = run_arm(wl, b, arm, min(args.micro, b), arena=arena, kv_bar=kv_bar)
+            print(json.dumps({"run": "sec5", "budget_GiB": budget / GiB, "arm": arm, "kv_bar": kv_bar, "batch": b,
+                              "result": res}), flush=True)
     else:
         for B, K in CFG5_SWEEP:
             wl = WORKLOADS["cfg5"].with_(B=B, K=K, name=f"cfg5_B{B}_K{K}")

@@ -76,6 +76,9 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
         if kind == "evict":
             cache.evict(evict_to, layer=layer)
             q = k = v = out = None
+        elif kind == "recent":                      # Algorithm 3's rule; `evict_to` pairs stay
+            cache.keep_most_recent(evict_to, layer=layer)
+            q = k = v = out = None
         else:
             q, k, v = inp.block(layer, pos0, I)
             if kind == "prefill":
@@ -89,7 +92,9 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
         stats["calls"] += 1
         for (smp, kh), unit in oracles.items():
             where = f"call {ci} ({kind} pos0={pos0} I={I}) unit ({smp},{kh})"
-            if kind != "evict":
+            if kind == "recent":
+                unit.keep_most_recent(evict_to)
+            elif kind != "evict":
                 ref = unit.process_block(_np(q[smp, :, kh * g:(kh + 1) * g]), _np(k[smp, :, kh]), _np(v[smp, :, kh]),
                                          pos0, -1)
                 err = float(np.abs(_np(out[smp, :, kh * g:(kh + 1) * g]) - ref).max())
@@ -98,7 +103,7 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
             want_rows = (ci % check_rows_every == 0) or ci == len(calls) - 1
             ids, sw, kr, vr = cache.export(layer, smp, kh, rows=want_rows)
             ids = ids.numpy().astype(np.int64)
-            if evict_to >= 0 and len(unit) > evict_to:
+            if kind != "recent" and evict_to >= 0 and len(unit) > evict_to:
                 check_kept(unit, ids, evict_to, stats, where)
             assert np.array_equal(ids, unit.kv_ids), f"{where}: kv_ids differ from the oracle's"
             n_gpu, cur = cache.length(layer, smp)

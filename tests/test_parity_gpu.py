@@ -135,6 +135,23 @@ def test_algorithm1_cadence_on_gpu():
     run_lockstep(wl, all_units(wl), calls=calls, growth=p, check_rows_every=3)
 
 
+@pytest.mark.parametrize("dtype,d,kv_bar", [("bf16", 128, 2), ("bf16", 128, 65), ("f32", 64, 5)])
+def test_extreme_decoding_arm_on_gpu(dtype, d, kv_bar):
+    # Algorithm 3: full cache during the prompt, then only the most recent pair survives each cut
+    s, gen = 200, 70
+    wl = tiny("ed", s=s, B=48, K=s, steps=gen, dtype=dtype, d=d, Hq=8, Hkv=2)
+    calls = [("prefill", t, min(48, s - t), -1) for t in range(0, s, 48)] + [("recent", 0, 0, 1)]
+    n = 1
+    for t in range(gen):
+        calls.append(("decode", s + t, 1, -1))
+        n += 1
+        if n == kv_bar:
+            calls.append(("recent", 0, 0, 1))
+            n = 1
+    st = run_lockstep(wl, all_units(wl), calls=calls, growth=kv_bar, check_rows_every=5)
+    assert st["calls"] == len(calls)
+
+
 # ------------------------------------------------------------------ API behaviour on the device
 def test_error_codes_and_state_tracking():
     wl = tiny("errors", dtype="bf16", d=128)
