@@ -23,6 +23,11 @@ Readings of points the paper leaves open (each is a convention of this build):
     Algorithm 1's literal decode-time curr_id (one larger) is available through
     the ``curr_id`` argument of :meth:`UnitCache.evict`.
   * ties in ave_weights: the pair with the lower position id is kept.
+  * left padding (Sec. 3: shorter prompts are padded on the left): a padding
+    position produces no attention row (its output is zero and it adds nothing
+    to sum_weights) and its pair is masked for every query, so its sum_weights
+    stays 0; padding pairs rank below every real pair at an eviction (the paper
+    does not say how padding meets eviction).
   * survivors keep their sum_weights (the vector is "variable-sized": entries
     leave with their pairs and nothing is reset).
 
@@ -47,9 +52,10 @@ class UnitCache:
     Sec. 3.2: ``kv_ids`` (position ids, ascending), ``sum_weights`` and the
     key/value rows themselves."""
 
-    def __init__(self, d: int, g: int = 1, scale: float | None = None):
+    def __init__(self, d: int, g: int = 1, scale: float | None = None, left_pad: int = 0):
         self.d = int(d)
         self.g = int(g)
+        self.left_pad = int(left_pad)  # positions 0 .. left_pad-1 of this sample are padding (Sec. 3)
         self.scale = (1.0 / math.sqrt(d)) if scale is None else float(scale)
         self.kv_ids = np.zeros(0, dtype=np.int64)
         self.k = np.zeros((0, d), dtype=np.float64)
@@ -88,21 +94,27 @@ class UnitCache:
 
         out = np.zeros((I, self.g, self.d))
         weights = np.zeros((I, self.g, n_old + I)) if return_weights else None
+        real = self.kv_ids >= self.left_pad          # padding pairs are masked for every query
+        n_real_queries = 0
         for i in range(I):
-            # visible pairs: every cached one, and the block's own up to position pos0 + i.
-            # kv_ids is ascending, so these are exactly the first m entries.
+            if pos0 + i < self.left_pad:
+                continue                             # a padding position: no output, no attention row
+            n_real_queries += 1
+            # visible pairs: every cached one, and the block's own up to position pos0 + i
+            # (kv_ids is ascending, so these are the first m entries), minus the padding pairs.
             m = n_old + i + 1
             assert self.kv_ids[m - 1] == pos0 + i
+            vis = np.nonzero(real[:m])[0]
             for h in range(self.g):
-                logits = self.scale * (self.k[:m] @ q[i, h])
+                logits = self.scale * (self.k[vis] @ q[i, h])
                 w = np.exp(logits - logits.max())
                 w = w / w.sum()                      # attn_weights[i] for this head
-                out[i, h] = w @ self.v[:m]
-                self.sum_weights[:m] += w            # sum_weights += attn_weights[i]
+                out[i, h] = w @ self.v[vis]
+                self.sum_weights[vis] += w           # sum_weights += attn_weights[i]
                 if return_weights:
-                    weights[i, h, :m] = w
+                    weights[i, h, vis] = w
         self.last_pos = pos0 + I - 1
-        self.rows_processed += I * self.g
+        self.rows_processed += n_real_queries * self.g
         if evict_to >= 0 and len(self) > evict_to:
             self.evict(evict_to)
         return (out, weights) if return_weights else out
@@ -126,7 +138,8 @@ class UnitCache:
     def evict(self, target: int, curr_id: int | None = None, kept_ids=None):
         """Remove the pairs with the smallest ave_weights until ``target`` remain.
 
-        Ranking: ave_weights descending, ties -> lower position id first; the first ``target``
+        Ranking: ave_weights descending, ties -> lower position id first (padding pairs of a
+        left-padded sample rank after every real pair); the first ``target``
         survive and stay in ascending position order (stable compaction).  ``kept_ids`` overrides
         the selection (used by lock-step parity to follow a choice made inside the tolerance
         band); the snapshot in ``last_eviction`` always holds the oracle's own choice.
@@ -136,7 +149,8 @@ class UnitCache:
         if target >= n:
             return None
         ave = self.ave_weights(curr_id)
-        order = np.lexsort((self.kv_ids, -ave))          # primary: -ave, secondary: id
+        # primary: real pairs before padding pairs (padding always leaves first), then -ave, then id
+        order = np.lexsort((self.kv_ids, -ave, self.kv_ids < self.left_pad))
         own_keep = np.sort(order[:target])
         cut = float(ave[order[target - 1]]) if target > 0 else math.inf
         snap = {
@@ -207,14 +221,15 @@ def _trace_entry(unit: UnitCache):
 
 
 def run_north_star(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec: int = 1,
-                   g: int | None = None, scale: float | None = None):
+                   g: int | None = None, scale: float | None = None, left_pad: int = 0):
     """Blocks of ``block`` prompt tokens (ragged tail allowed), the cache cut back to ``kv_max``
     after every block; then ``steps`` decode steps, cut back to ``kv_max`` whenever the cache
-    has grown to ``kv_max + p_dec``.   q: (s+steps, g, d); k, v: (s+steps, d).
+    has grown to ``kv_max + p_dec``.   q: (s+steps, g, d); k, v: (s+steps, d); the first
+    ``left_pad`` positions are padding.
     Returns (outputs (s+steps, g, d), trace of kv_ids after every call, unit)."""
     q = np.asarray(q, dtype=np.float64)
     g = q.shape[1] if g is None else g
-    unit = UnitCache(q.shape[2], g, scale)
+    unit = UnitCache(q.shape[2], g, scale, left_pad)
     outs, trace = [], []
     pos = 0
     while pos < s:

@@ -496,3 +496,76 @@ def test_keep_most_recent_keeps_ids_and_sums_of_the_tail():
         assert np.array_equal(a[6:], b)
     u.keep_most_recent(5)                       # nothing to remove
     assert len(u) == 3
+
+
+# ---------------------------------------------------------------- left padding (Sec. 3)
+@pytest.mark.parametrize("pad,block", [(1, 4), (7, 4), (8, 8), (13, 5), (19, 32)])
+def test_left_padding_full_cache_equals_dense_attention_over_the_real_tokens(pad, block):
+    # nothing is evicted: the real queries must see exactly the un-padded sequence, whatever sits in the padding
+    s, g, d = 29, 2, 8
+    q, k, v = rand_qkv(41, s, g, d)
+    out, _, unit = run_north_star(q, k, v, s, block, kv_max=1000, steps=0, left_pad=pad)
+    np.testing.assert_allclose(out[pad:], dense_causal_attention(q[pad:], k[pad:], v[pad:]), atol=1e-12)
+    assert np.all(out[:pad] == 0.0)
+    assert np.all(unit.sum_weights[:pad] == 0.0)
+    _, _, ref = run_north_star(q[pad:], k[pad:], v[pad:], s - pad, block, kv_max=1000, steps=0)
+    np.testing.assert_allclose(unit.sum_weights[pad:], ref.sum_weights, rtol=1e-12)
+    assert unit.rows_processed == g * (s - pad)
+
+
+@pytest.mark.parametrize("pad_blocks", [1, 2])
+@pytest.mark.parametrize("g", [1, 3])
+def test_left_padding_by_whole_blocks_is_the_unpadded_run_shifted(pad_blocks, g):
+    # padding fills the first blocks exactly, so block boundaries and every eviction line up with the run on the
+    # real tokens alone: same outputs, same survivors (ids shifted by the padding), same sums
+    s, B, K, steps, d = 48, 8, 5, 6, 4
+    pad = pad_blocks * B
+    q, k, v = rand_qkv(43, s + steps, g, d)
+    out, trace, unit = run_north_star(q, k, v, s, B, K, steps, left_pad=pad)
+    out0, trace0, unit0 = run_north_star(q[pad:], k[pad:], v[pad:], s - pad, B, K, steps)
+    np.testing.assert_allclose(out[pad:], out0, atol=1e-12)
+    assert np.array_equal(unit.kv_ids - pad, unit0.kv_ids)
+    np.testing.assert_allclose(unit.sum_weights, unit0.sum_weights, rtol=1e-12)
+    for ids, ids0 in zip(trace[pad_blocks + 1:], trace0[1:]):     # once one real block went through, padding is gone
+        assert np.array_equal(np.asarray(ids) - pad, ids0)
+
+
+def test_left_padding_leaves_first_and_from_the_top():
+    s, B, K, g, d, pad = 40, 8, 12, 2, 4, 11
+    q, k, v = rand_qkv(47, s, g, d)
+    unit = UnitCache(d, g, left_pad=pad)
+    for pos in range(0, s, B):
+        before = set(unit.kv_ids.tolist()) | set(range(pos, pos + B))
+        unit.process_block(q[pos:pos + B], k[pos:pos + B], v[pos:pos + B], pos, K)
+        kept = set(unit.kv_ids.tolist())
+        gone = before - kept
+        pads_kept = sorted(i for i in kept if i < pad)
+        if any(i >= pad for i in gone):
+            assert not pads_kept                           # a real pair left only once all padding was gone
+        assert pads_kept == list(range(len(pads_kept)))    # the padding that stays is the lowest positions
+        assert np.all(unit.sum_weights[unit.kv_ids < pad] == 0.0)
+    assert unit.sum_weights.sum() + unit.evicted_mass == pytest.approx(g * (s - pad), rel=1e-12)
+
+
+def test_left_padding_masked_dense_replay():
+    # outputs recomputed from the trace of visible ids over the original arrays, padding positions removed
+    s, B, K, steps, g, d, pad = 37, 6, 7, 5, 2, 4, 9
+    q, k, v = rand_qkv(53, s + steps, g, d)
+    out, trace, _ = run_north_star(q, k, v, s, B, K, steps, left_pad=pad)
+    scale = 1.0 / math.sqrt(d)
+    cached, pos, call = [], 0, 0
+    bounds = [(p0, min(B, s - p0)) for p0 in range(0, s, B)] + [(s + t, 1) for t in range(steps)]
+    for p0, I in bounds:
+        for i in range(I):
+            qi = p0 + i
+            if qi < pad:
+                assert np.all(out[qi] == 0.0)
+                continue
+            js = [j for j in list(cached) + list(range(p0, qi + 1)) if j >= pad]
+            for h in range(g):
+                lg = np.array([scale * float(q[qi, h] @ k[j]) for j in js])
+                w = np.exp(lg - lg.max())
+                w /= w.sum()
+                np.testing.assert_allclose(out[qi, h], sum(wj * v[j] for wj, j in zip(w, js)), atol=1e-12)
+        cached = list(trace[call])
+        call += 1
