@@ -181,6 +181,18 @@ bm_status_t bm_decode_step_host(bm_cache_t* cache, int32_t layer, int32_t sample
                                 void* out /*HOST*/, int32_t evict_to, void* staging /*DEVICE*/,
                                 size_t staging_bytes, void* cuda_stream);
 
+/* ---- left-padded samples (Sec. 3: prompts of unequal length are padded on the left) ----
+ * pads[s] = number of padding positions at the start of sample s (HOST array of cfg.batch entries; NULL or
+ * all zeros switches padding off).  From then on, for sample s: a pair whose position id is below pads[s] is
+ * masked for every real query, so its sum_weights stays 0, and it ranks below every real pair at an eviction
+ * (padding leaves first, highest position first); a query at a padding position produces an all-zero output
+ * row and adds nothing to sum_weights.  Padding pairs occupy cache rows like any other pair until they are
+ * evicted, so n stays equal over the samples of a call.  The paper does not say how padding meets eviction;
+ * this is the build's reading.  Must be called while every cache of the handle is empty, else BM_ERR_STATE;
+ * negative entries give BM_ERR_INVALID.  The copy to the device is ordered on cuda_stream, like the calls
+ * that use it. */
+bm_status_t bm_cache_set_left_pad(bm_cache_t* cache, const int32_t* pads /*HOST*/, void* cuda_stream);
+
 /* ---- state access ---- */
 /* Host mirror of n and curr_id (-1 when empty) of one (layer, sample); no synchronisation. */
 bm_status_t bm_cache_len(const bm_cache_t* cache, int32_t layer, int32_t sample, int32_t* n /*HOST out*/,

@@ -48,6 +48,7 @@ SIGNATURES = {
     "bm_decode_step": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp]),
     "bm_evict": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp]),
     "bm_keep_most_recent": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp]),
+    "bm_cache_set_left_pad": (_i32, [_vp, _vp, _vp]),
     "bm_staging_bytes": (_i32, [_cfgp, _i32, _i32, C.POINTER(_sz)]),
     "bm_prefill_block_host": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
     "bm_decode_step_host": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp, _sz, _vp]),
@@ -258,6 +259,17 @@ class BatchMaxCache:
         """Algorithm 3's rule: all but the `keep` most recent pairs leave the cache."""
         ns = self.cfg.batch - sample0 if nsamples is None else nsamples
         _check(lib().bm_keep_most_recent(self.h, layer, sample0, ns, keep, _stream(stream)), "bm_keep_most_recent")
+
+    def set_left_pad(self, pads, stream=None):
+        """pads[s] = padding positions at the start of sample s (a sequence of cfg.batch ints, or None)."""
+        if pads is None:
+            _check(lib().bm_cache_set_left_pad(self.h, None, _stream(stream)), "bm_cache_set_left_pad")
+            return
+        pads = [int(x) for x in pads]
+        assert len(pads) == self.cfg.batch
+        arr = (C.c_int32 * len(pads))(*pads)
+        _check(lib().bm_cache_set_left_pad(self.h, C.cast(arr, C.c_void_p), _stream(stream)),
+               "bm_cache_set_left_pad")
 
     # -- host-fed variants ---------------------------------------------------------------------------
     def _stage(self, ns, I):

@@ -81,6 +81,7 @@ size_t ws_lse_bytes(const bm_config_t* c) {
 size_t ws_newsum_bytes(const bm_config_t* c) {
   return align_up(sizeof(float) * (size_t)call_samples(c) * c->n_kv_heads * c->block_max, 256);
 }
+size_t ws_pad_bytes(const bm_config_t* c) { return align_up(sizeof(int32_t) * (size_t)c->batch, 256); }
 
 }  // namespace
 
@@ -96,6 +97,8 @@ struct bm_cache {
   int32_t* status;
   float* ws_lse;
   float* ws_new_sum;
+  int32_t* left_pad = nullptr;   // [batch] device copy of the samples' padding counts (in the workspace)
+  bool has_pad = false;          // some sample is left-padded
   std::vector<int32_t> n, curr_id;  // [L * b] host mirror
   // host-fed calls run as a three-stage pipeline on streams owned by the handle -- input copies, the pass,
   // the output copy -- so that the three stages of consecutive calls overlap (PCIe is full duplex); the
@@ -148,6 +151,7 @@ CacheView make_view(const bm_cache* c, int layer, int sample0, int nsamples, int
   v.g = c->g;
   v.nsamples = nsamples;
   v.status = c->status;
+  v.left_pad = c->has_pad ? c->left_pad + sample0 : nullptr;
   return v;
 }
 
@@ -182,7 +186,7 @@ bm_status_t bm_max_batch(const bm_config_t* cfg, size_t hbm_budget_bytes, int32_
 
 bm_status_t bm_workspace_bytes(const bm_config_t* cfg, size_t* bytes) {
   if (!config_ok(cfg, true) || bytes == nullptr) return BM_ERR_INVALID;
-  *bytes = ws_lse_bytes(cfg) + ws_newsum_bytes(cfg);
+  *bytes = ws_lse_bytes(cfg) + ws_newsum_bytes(cfg) + ws_pad_bytes(cfg);
   return BM_OK;
 }
 
@@ -217,6 +221,7 @@ bm_status_t bm_cache_create(const bm_config_t* cfg, void* arena, size_t arena_by
   if (off > need_arena) { delete c; return BM_ERR_OOM; }
   c->ws_lse = static_cast<float*>(workspace);
   c->ws_new_sum = reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_lse_bytes(cfg));
+  c->left_pad = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + ws_lse_bytes(cfg) + ws_newsum_bytes(cfg));
   c->n.assign((size_t)cfg->n_layers * cfg->batch, 0);
   c->curr_id.assign((size_t)cfg->n_layers * cfg->batch, -1);
   // Unwritten rows are read as zero-weight padding by the tiled kernels, so they must hold finite values.
@@ -481,6 +486,30 @@ bm_status_t bm_cache_len(const bm_cache_t* c, int32_t layer, int32_t sample, int
   const size_t o = (size_t)layer * c->cfg.batch + sample;
   *n = c->n[o];
   if (curr_id != nullptr) *curr_id = c->curr_id[o];
+  return BM_OK;
+}
+
+bm_status_t bm_cache_set_left_pad(bm_cache_t* c, const int32_t* pads, void* cuda_stream) {
+  if (c == nullptr) return BM_ERR_INVALID;
+  for (int v : c->n)
+    if (v != 0) return BM_ERR_STATE;
+  for (int v : c->curr_id)
+    if (v != -1) return BM_ERR_STATE;
+  bool any = false;
+  if (pads != nullptr)
+    for (int s = 0; s < c->cfg.batch; ++s) {
+      if (pads[s] < 0) return BM_ERR_INVALID;
+      any = any || pads[s] > 0;
+    }
+  c->has_pad = any;
+  if (!any) return BM_OK;
+  bm_status_t st = set_device(c);
+  if (st != BM_OK) return st;
+  ++c->dev_calls;
+  // the source may be pageable: the runtime stages it before this call returns
+  if (cudaMemcpyAsync(c->left_pad, pads, sizeof(int32_t) * (size_t)c->cfg.batch, cudaMemcpyHostToDevice,
+                      static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return BM_ERR_CUDA;
   return BM_OK;
 }
 

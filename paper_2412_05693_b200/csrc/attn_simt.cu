@@ -81,8 +81,10 @@ __global__ void __launch_bounds__(kThreads) attn_fwd_simt(CacheView c, BlockArgs
   float* sM = sS + kTile * (kTile + 1);
   float* sL = sM + kTile;
   float* sAl = sL + kTile;
+  int* sKp = reinterpret_cast<int*>(sAl + kTile);   // [64] 1 = the tile's key is a padding pair
 
   const int unit = blockIdx.y, smp = unit / c.Hkv, kh = unit % c.Hkv;
+  const int pad = sample_left_pad(c, smp);
   const int R = a.I * c.g, row0 = blockIdx.x * kTile;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4, lane = tid & 31, warp = tid >> 5;
 
@@ -100,6 +102,13 @@ __global__ void __launch_bounds__(kThreads) attn_fwd_simt(CacheView c, BlockArgs
   for (int j0 = 0; j0 < n_keys; j0 += kTile) {
     __syncthreads();  // previous iteration finished with sKV / sS
     load_tile<T, D>(sKV, tid, [&](int r) { return key_row_ptr<T, D>(c, c.k_slab, a.k, unit, smp, kh, a.I, j0 + r); });
+    if (tid < kTile) {
+      const int j = j0 + tid;
+      int is_pad = 0;
+      if (pad > 0 && j < c.n_old + a.I)
+        is_pad = (j < c.n_old ? c.kv_ids[(size_t)unit * c.cap + j] : a.pos0 + (j - c.n_old)) < pad;
+      sKp[tid] = is_pad;
+    }
     __syncthreads();
     float acc[4][4];
     dot_tile<D>(sQ, sKV, ty, tx, acc);
@@ -113,7 +122,10 @@ __global__ void __launch_bounds__(kThreads) attn_fwd_simt(CacheView c, BlockArgs
     for (int rr = 0; rr < 8; ++rr) {
       const int r = warp * 8 + rr, row = row0 + r;
       const int vis = (row < R) ? (c.n_old + row / c.g + 1) : 1;
-      const bool ok0 = (j0 + lane) < vis, ok1 = (j0 + lane + 32) < vis;
+      // a real query does not see padding pairs; a padding query's row is computed over everything and dropped
+      const bool real = (row < R) && (a.pos0 + row / c.g >= pad);
+      const bool ok0 = (j0 + lane) < vis && !(real && sKp[lane]);
+      const bool ok1 = (j0 + lane + 32) < vis && !(real && sKp[lane + 32]);
       const float s0 = ok0 ? sS[r * (kTile + 1) + lane] : -INFINITY;
       const float s1 = ok1 ? sS[r * (kTile + 1) + lane + 32] : -INFINITY;
       float mt = fmaxf(s0, s1);
@@ -158,11 +170,12 @@ __global__ void __launch_bounds__(kThreads) attn_fwd_simt(CacheView c, BlockArgs
     const int r = ty + 16 * x, row = row0 + r;
     if (row >= R) continue;
     const int i = row / c.g, h = row % c.g;
-    const float inv = 1.f / sL[r];
+    const bool real = a.pos0 + i >= pad;          // a padding query: zero output, and +inf so that it has no weights
+    const float inv = real ? 1.f / sL[r] : 0.f;
     T* op = reinterpret_cast<T*>(a.out) + ((size_t)(smp * a.I + i) * c.Hq + kh * c.g + h) * D;
 #pragma unroll
     for (int y = 0; y < D / 16; ++y) op[tx + 16 * y] = Elem<T>::to_out(o[x][y] * inv);
-    if (tx == 0) a.lse[(size_t)unit * R + row] = sM[r] + logf(sL[r]);
+    if (tx == 0) a.lse[(size_t)unit * R + row] = real ? sM[r] + logf(sL[r]) : INFINITY;
   }
 }
 
@@ -216,6 +229,9 @@ __global__ void __launch_bounds__(kThreads) score_simt(CacheView c, BlockArgs a)
       float tot = 0.f;
 #pragma unroll
       for (int t = 0; t < 16; ++t) tot += sRed[t * kTile + tid];
+      const int pad = sample_left_pad(c, smp);
+      if (pad > 0 && (j < c.n_old ? c.kv_ids[(size_t)unit * c.cap + j] : a.pos0 + (j - c.n_old)) < pad)
+        tot = 0.f;                                  // a padding pair is masked for every query
       if (j < c.n_old) c.sum_weights[(size_t)unit * c.cap + j] += tot;
       else a.new_sum[(size_t)unit * a.I + (j - c.n_old)] = tot;
     }
@@ -224,7 +240,7 @@ __global__ void __launch_bounds__(kThreads) score_simt(CacheView c, BlockArgs a)
 
 template <typename T, int D>
 cudaError_t launch_attn_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
-  const size_t smem = sizeof(float) * (2 * kTile * (D + 1) + kTile * (kTile + 1) + 3 * kTile);
+  const size_t smem = sizeof(float) * (2 * kTile * (D + 1) + kTile * (kTile + 1) + 4 * kTile);
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(attn_fwd_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

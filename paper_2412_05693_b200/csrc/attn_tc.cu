@@ -41,6 +41,10 @@ struct TcArgs {
   float* new_sum;
   int cap;
   int* status;
+  // left-padded samples: padding counts of the range's samples (null: none), cached ids, the block's first position
+  const int* left_pad;
+  const int* kv_ids;
+  int pos0;
 };
 
 // ------------------------------------------------------------------------------------------------------
@@ -62,7 +66,8 @@ struct FwdSmem {
   static constexpr int kThreads = 128 * NT + 64;
 };
 
-template <int D, int NT>
+// PAD: the range has left-padded samples (a separate instance, so that the common case carries none of its masks).
+template <int D, int NT, bool PAD>
 __global__ void __launch_bounds__(128 * NT + 64, NT == 2 ? 1 : 2)
 attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   using L = FwdSmem<D, NT>;
@@ -76,6 +81,7 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::kBars);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* np_slot = reinterpret_cast<int*>(tmem_slot + 2);   // [2] cached padding pairs, counted per query tile
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int unit = blockIdx.y, smp = unit / a.Hkv, kh = unit % a.Hkv;
@@ -116,6 +122,8 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   };
   if (warp == kTmaWarp && lane == 0) {
     *abort_flag = 0;
+    np_slot[0] = 0;
+    np_slot[1] = 0;
     for (int x = 0; x < 2; ++x) {
       mbar_init(&bars[B_QFULL + x], 1);
       mbar_init(&bars[B_SFULL + x], 1);
@@ -208,14 +216,35 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
       const uint32_t lane_addr = (uint32_t)(quad * 32) << 16;
       const int row = row0[x] + r;
       const int i_row = min(a.I - 1, i0[x] + r / a.g);  // rows past the block's end behave like its last input
+      // Left-padded sample: the cached padding pairs are the first n_pad rows (ids ascend), counted here by the
+      // tile's 128 threads; a real query masks them and the block's padding positions, a padding query is
+      // computed over everything and dropped in the epilogue.
+      int pad = 0, n_pad = 0;
+      if (PAD) {
+        pad = a.left_pad[smp];
+        const int* ids = a.kv_ids + (size_t)unit * a.cap;
+        if (pad > 0 && a.n_old > 0 && ids[0] < pad) {          // uniform over the tile's threads
+          int cnt = 0;
+          for (int t = r; t < min(a.n_old, pad); t += 128) cnt += ids[t] < pad;
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+          if (lane == 0 && cnt > 0) atomicAdd(&np_slot[x], cnt);
+          named_bar_sync(1 + x, 128);
+          n_pad = np_slot[x];
+        }
+      }
+      const bool real_row = !PAD || a.pos0 + i_row >= pad;
       float m_used = -INFINITY, l = 0.f;
       for (int j = 0; j < T[x]; ++j) {
         mbar_wait(&bars[B_SFULL + x], j & 1, abort_flag, a.status);
         tc_fence_after();
-        // visible columns of this key tile for this row
+        // visible columns of this key tile for this row: [nlo, nvis)
         const int nvis = (j < t_old) ? min(kTileN, a.n_old - j * kTileN)
                                      : max(0, min(kTileN, i_row - (j - t_old) * kTileN + 1));
-        const bool full = __all_sync(0xffffffffu, nvis >= kTileN);   // warp-uniform: nothing to mask in this tile
+        const int nlo = (!PAD || !real_row) ? 0
+                        : (j < t_old) ? max(0, min(kTileN, n_pad - j * kTileN))
+                                      : max(0, min(kTileN, pad - a.pos0 - (j - t_old) * kTileN));
+        const bool full = __all_sync(0xffffffffu, nvis >= kTileN && nlo == 0);   // warp-uniform: nothing to mask
         float mx = -INFINITY;
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {                              // two TMEM loads in flight
@@ -232,8 +261,8 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
           } else {
 #pragma unroll
             for (int e = 0; e < 32; ++e) {
-              mx = fmaxf(mx, (hh * 64 + e < nvis) ? __uint_as_float(ra[e]) : -INFINITY);
-              mx = fmaxf(mx, (hh * 64 + 32 + e < nvis) ? __uint_as_float(rb[e]) : -INFINITY);
+              mx = fmaxf(mx, (hh * 64 + e < nvis && hh * 64 + e >= nlo) ? __uint_as_float(ra[e]) : -INFINITY);
+              mx = fmaxf(mx, (hh * 64 + 32 + e < nvis && hh * 64 + 32 + e >= nlo) ? __uint_as_float(rb[e]) : -INFINITY);
             }
           }
         }
@@ -271,8 +300,8 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
             float p0 = ex2(x0), p1 = ex2(x1);
             if (!full) {
               const int c0 = cc * 32 + 2 * e;
-              p0 = (c0 < nvis) ? p0 : 0.f;
-              p1 = (c0 + 1 < nvis) ? p1 : 0.f;
+              p0 = (c0 < nvis && c0 >= nlo) ? p0 : 0.f;
+              p1 = (c0 + 1 < nvis && c0 + 1 >= nlo) ? p1 : 0.f;
             }
             ps0 += p0;
             ps1 += p1;
@@ -294,7 +323,7 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
       // epilogue: O / l -> bf16 -> swizzled tile in the (now idle) query buffer -> TMA store; log2-sum-exp
       mbar_wait(&bars[B_ODONE + x], (T[x] - 1) & 1, abort_flag, a.status);
       tc_fence_after();
-      const float inv = 1.f / l;
+      const float inv = real_row ? 1.f / l : 0.f;     // a padding query's output row is zero
       unsigned char* stage = sm + L::kQ + x * L::kTileBytes;
 #pragma unroll
       for (int cc = 0; cc < D / 32; ++cc) {
@@ -312,7 +341,7 @@ attn_fwd_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
           *reinterpret_cast<uint4*>(stage + (piece >> 3) * 16384 + sw128_offset(r, piece & 7)) = w;
         }
       }
-      if (row < R) a.lse2[(size_t)unit * R + row] = m_used + log2f(l);
+      if (row < R) a.lse2[(size_t)unit * R + row] = real_row ? m_used + log2f(l) : INFINITY;  // +inf: no weights
       fence_async_smem();
       named_bar_sync(1 + x, 128);
       if (r == 0) {
@@ -490,6 +519,11 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
 #pragma unroll
       for (int w = 0; w < kScoreWG; ++w) tot += sPart[w * 128 + key];   // fixed order
       const int j = is_old ? kt * kTileN + key : c0 + key;
+      if (a.left_pad != nullptr) {                  // a padding pair is masked for every query
+        const int pad = a.left_pad[smp];
+        const bool in_range = is_old ? j < a.n_old : j < a.I;
+        if (pad > 0 && in_range && (is_old ? a.kv_ids[(size_t)unit * a.cap + j] : a.pos0 + j) < pad) tot = 0.f;
+      }
       if (is_old) { if (j < a.n_old) a.sum_weights[(size_t)unit * a.cap + j] += tot; }
       else if (j < a.I) a.new_sum[(size_t)unit * a.I + j] = tot;
     }
@@ -561,6 +595,7 @@ TcArgs make_args(const CacheView& c, const BlockArgs& a) {
   t.scale_log2 = a.scale * kLog2e;
   t.lse2 = a.lse; t.sum_weights = c.sum_weights; t.new_sum = a.new_sum;
   t.cap = c.cap; t.status = c.status;
+  t.left_pad = c.left_pad; t.kv_ids = c.kv_ids; t.pos0 = a.pos0;
   return t;
 }
 
@@ -568,19 +603,20 @@ TcArgs make_args(const CacheView& c, const BlockArgs& a) {
 TcMaps g_maps;
 const void* g_maps_q = nullptr;
 
-template <int D, int NT>
+template <int D, int NT, bool PAD>
 cudaError_t launch_fwd_nt(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
   using L = FwdSmem<D, NT>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc<D, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc<D, NT, PAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         L::kTotal);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   const int R = a.I * c.g;
   dim3 grid((R + NT * kTileM - 1) / (NT * kTileM), c.nsamples * c.Hkv);
   ProfileScope prof(kAttnFwd, st);
-  attn_fwd_tc<D, NT><<<grid, L::kThreads, L::kTotal, st>>>(g_maps, make_args(c, a));
+  attn_fwd_tc<D, NT, PAD><<<grid, L::kThreads, L::kTotal, st>>>(g_maps, make_args(c, a));
   count_launch();
   return cudaGetLastError();
 }
@@ -592,7 +628,9 @@ int g_fwd_tiles_override = 0;
 
 template <int D>
 cudaError_t launch_fwd_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
-  return g_fwd_tiles_override == 2 ? launch_fwd_nt<D, 2>(c, a, st) : launch_fwd_nt<D, 1>(c, a, st);
+  if (c.left_pad != nullptr)
+    return g_fwd_tiles_override == 2 ? launch_fwd_nt<D, 2, true>(c, a, st) : launch_fwd_nt<D, 1, true>(c, a, st);
+  return g_fwd_tiles_override == 2 ? launch_fwd_nt<D, 2, false>(c, a, st) : launch_fwd_nt<D, 1, false>(c, a, st);
 }
 
 template <int D>

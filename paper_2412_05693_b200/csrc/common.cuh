@@ -18,7 +18,14 @@ struct CacheView {
   int32_t Hq, Hkv, g;
   int32_t nsamples;
   int32_t* status;     // device status word
+  const int32_t* left_pad;  // [nsamples] padding positions at the start of each sample of the range, or null
 };
+
+// Left padding (Sec. 3): positions below the sample's count are padding.  A padding pair is masked for every
+// real query; a padding query produces a zero output row and no attention weights.
+__device__ inline int sample_left_pad(const CacheView& c, int smp) {
+  return c.left_pad != nullptr ? c.left_pad[smp] : 0;
+}
 
 // One forward pass over a block (I inputs) for the range.
 struct BlockArgs {

@@ -80,6 +80,10 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
   T* vslab = reinterpret_cast<T*>(c.v_slab) + base * D;
   const bool evict_one = (a.target == n1 - 1);
   const bool evict_general = (a.target >= 0 && a.target < n1 - 1);
+  // left-padded sample: padding pairs are masked and leave first; a query at a padding position (not a real
+  // decode step) gets a zero output and no weights
+  const int pad = sample_left_pad(c, smp);
+  const bool q_real = a.pos >= pad;
 
   // queries of the group -> smem (fp32); the step's pair -> row n_old of the cache
   for (int t = tid; t < G * D; t += kDecThreads) {
@@ -135,8 +139,9 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
 #pragma unroll
           for (int h = 0; h < G; ++h) dot[h] += __shfl_xor_sync(0xffffffffu, dot[h], off);
         if (lr == 0 && j < n1) {
+          const bool masked = q_real && s.id[j] < pad;
 #pragma unroll
-          for (int h = 0; h < G; ++h) s.p[h * n1p + j] = dot[h] * sc2;
+          for (int h = 0; h < G; ++h) s.p[h * n1p + j] = masked ? -INFINITY : dot[h] * sc2;
         }
       }
     }
@@ -176,7 +181,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
     float t = 0.f;
 #pragma unroll
     for (int w = 0; w < kDecWarps; ++w) t += s.wred[(G + h) * kDecWarps + w];  // fixed order
-    sm[h] = 1.f / t;
+    sm[h] = q_real ? 1.f / t : 0.f;
   }
   (void)mx;
 
@@ -194,7 +199,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
     const float sw = ((j < c.n_old) ? c.sum_weights[base + j] : 0.f) + add;
     s.score[j] = sw;
     if (evict_one) {
-      const float ave = sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
+      const float ave = s.id[j] < pad ? -1.f : sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
       if (ave <= best_ave) { best_ave = ave; best_j = j; }   // j ascends: ties move to the higher position
     } else {
       c.sum_weights[base + j] = sw;

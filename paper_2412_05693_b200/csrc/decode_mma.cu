@@ -187,6 +187,17 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
   // ---- softmax statistics over the n1 rows with one barrier: every thread folds its own logits into a
   // (maximum, sum of exp2 relative to that maximum) pair per head, pairs are merged across the warp by shuffles
   // and across warps through shared memory in a fixed order.
+  // left-padded sample: padding pairs are masked and leave first (each thread masks the rows whose ids it
+  // loaded itself); a query at a padding position, which no real decode step is, gets zero output and no weights
+  const int pad = sample_left_pad(c, smp);
+  const bool q_real = a.pos >= pad;
+  if (pad > 0 && q_real) {
+    for (int j = tid; j < n1; j += kThreads)
+      if (s.id[j] < pad) {
+#pragma unroll
+        for (int h = 0; h < G; ++h) s.p[h * n1t + j] = -INFINITY;
+      }
+  }
   float inv[G], mfin[G];
   {
     float m[G], t[G];
@@ -229,7 +240,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
         tt += (mw == -INFINITY) ? 0.f : s.wred[(G + h) * kWarps + w] * ex2f(mw - mm);
       }
       mfin[h] = mm;
-      inv[h] = 1.f / tt;
+      inv[h] = q_real ? 1.f / tt : 0.f;
     }
   }
 
@@ -259,7 +270,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
     const float sw = old_sw + add;
     s.score[j] = sw;
     if (evict_one) {
-      const float ave = sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
+      const float ave = s.id[j] < pad ? -1.f : sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
       if (ave <= best_ave) { best_ave = ave; best_j = j; }   // j ascends: ties move to the higher position
     } else {
       c.sum_weights[base + j] = sw;

@@ -71,9 +71,12 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
   }
   __syncthreads();
   const float gf = (float)c.g;
+  const int pad = sample_left_pad(c, smp);
   auto ave_bits = [&](int j) -> uint32_t {
     const float cnt = (float)(e.curr_id + 1 - s.id[j]);
-    return __float_as_uint(s.score[j] / (gf * cnt));  // ave >= 0, so the bit pattern orders like the value
+    const uint32_t b = __float_as_uint(s.score[j] / (gf * cnt));  // ave >= 0: the bit pattern orders like the value
+    if (pad == 0) return b;
+    return s.id[j] < pad ? 0u : max(b, 1u);   // padding pairs rank below every real pair (left-padded samples)
   };
 
   if (target >= n_c) {

@@ -38,16 +38,24 @@ def check_kept(unit: UnitCache, gpu_ids: np.ndarray, target: int, stats: dict, w
     GPU's set when it differs inside the band)."""
     ave = unit.ave_weights()
     cand = unit.kv_ids
-    order = np.lexsort((cand, -ave))
-    cut = ave[order[target - 1]]
+    is_pad = cand < unit.left_pad                 # padding pairs of a left-padded sample rank after every real pair
+    order = np.lexsort((cand, -ave, is_pad))
+    n_real = int((~is_pad).sum())
     gpu = np.asarray(gpu_ids, dtype=np.int64)
     assert gpu.shape[0] == target, f"{where}: kept {gpu.shape[0]} != target {target}"
     assert np.all(np.diff(gpu) > 0), f"{where}: kept ids not ascending"
     in_cand = np.isin(gpu, cand)
     assert in_cand.all(), f"{where}: kept ids that were never candidates: {gpu[~in_cand][:8]}"
     kept_mask = np.isin(cand, gpu)
-    must_keep = ave > cut * (1 + BAND)
-    must_drop = ave < cut * (1 - BAND)
+    if target <= n_real:                          # the cut falls among the real pairs; all padding leaves
+        cut = ave[order[target - 1]]
+        must_keep = ~is_pad & (ave > cut * (1 + BAND))
+        must_drop = is_pad | (ave < cut * (1 - BAND))
+    else:                                         # every real pair stays, with the lowest padding positions
+        lowest = np.zeros_like(is_pad)
+        lowest[order[n_real:target]] = True
+        must_keep = ~is_pad | lowest
+        must_drop = is_pad & ~lowest
     assert not np.any(must_keep & ~kept_mask), f"{where}: dropped a pair clearly above the cut"
     assert not np.any(must_drop & kept_mask), f"{where}: kept a pair clearly below the cut"
     own = cand[np.sort(order[:target])]
@@ -58,15 +66,17 @@ def check_kept(unit: UnitCache, gpu_ids: np.ndarray, target: int, stats: dict, w
 
 
 def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=None, check_rows_every: int = 8,
-                 growth: int | None = None, sum_rtol: float | None = None):
+                 growth: int | None = None, sum_rtol: float | None = None, pads=None):
     """Run `calls` (default: the workload's spec schedule) on the GPU for the whole batch and on the
     oracle for `units` = [(sample, kv_head), ...].  Returns a dict of statistics; raises on any mismatch."""
     dev = torch.device("cuda", device)
     inp = Inputs(wl, dev)
     cfg = make_config(wl, device, growth)
     cache = BatchMaxCache(cfg)
+    if pads is not None:                            # left-padded samples: pads[sample] padding positions
+        cache.set_left_pad(pads)
     g = wl.g
-    oracles = {u: UnitCache(wl.d, g) for u in units}
+    oracles = {u: UnitCache(wl.d, g, left_pad=0 if pads is None else pads[u[0]]) for u in units}
     stats = {"adoptions": 0, "evictions": 0, "max_out_err": 0.0, "max_sum_rel": 0.0, "calls": 0, "tc_calls": 0}
     tol = OUT_TOL[wl.dtype]
     sum_rtol = sum_rtol if sum_rtol is not None else (2e-3 if wl.dtype == "bf16" else 2e-4)

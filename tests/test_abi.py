@@ -66,7 +66,8 @@ def test_max_batch_under_budget_and_pd_vs_decode_only_ratio():
 
 def test_workspace_and_staging_sizes():
     cfg = llama_cfg(max_call_samples=4)
-    assert bm.workspace_bytes(cfg) == 4 * (4 * 32 * 512 + 4 * 8 * 512)
+    # log-sum-exp of the query rows + column sums of the new pairs (per call) + one padding count per sample
+    assert bm.workspace_bytes(cfg) == 4 * (4 * 32 * 512 + 4 * 8 * 512) + 256
     assert binding.staging_bytes(cfg, 2, 512) == 2 * (2 * 512 * 32 * 128 * 2) + 2 * (2 * 512 * 8 * 128 * 2)
 
 

@@ -152,6 +152,46 @@ def test_extreme_decoding_arm_on_gpu(dtype, d, kv_bar):
     assert st["calls"] == len(calls)
 
 
+# ------------------------------------------------------------------ left-padded samples (Sec. 3)
+@pytest.mark.parametrize("dtype,d,s,B,K,pads", [
+    ("f32", 64, 200, 48, 40, [0, 37, 150]),         # SIMT path; padding inside a block and over whole blocks
+    ("bf16", 128, 640, 128, 160, [0, 70, 300]),     # tensor-core path; a whole 128-key tile of cached padding
+    ("bf16", 128, 640, 256, 96, [5, 255, 256]),     # padding ending at / just before a block boundary
+    ("bf16", 64, 300, 64, 64, [299, 1, 128]),       # one sample almost entirely padding
+])
+def test_left_padded_samples_lockstep(dtype, d, s, B, K, pads):
+    wl = tiny("leftpad", b=3, s=s, B=B, K=K, steps=6, dtype=dtype, d=d, Hq=8, Hkv=2)
+    st = run_lockstep(wl, all_units(wl), pads=pads, check_rows_every=2)
+    assert st["evictions"] > 0
+    if dtype == "bf16":
+        assert st["tc_calls"] == -(-s // B)          # every prefill call took the tensor-core kernels
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_left_padding_still_cached_during_decoding(dtype, d):
+    # prompt shorter than the limit: the padding is still cached when decoding starts, is masked there, and is
+    # what the first evicting decode steps remove (highest padding position first)
+    wl = tiny("leftpad_dec", b=3, s=50, B=32, K=60, steps=24, dtype=dtype, d=d, Hq=8, Hkv=2)
+    st = run_lockstep(wl, all_units(wl), pads=[0, 7, 30], check_rows_every=3)
+    assert st["evictions"] >= 3 * 2 * 10
+
+
+def test_left_pad_setter_errors():
+    wl = tiny("leftpad_err", dtype="bf16", d=128)
+    cache = bm.BatchMaxCache(make_config(wl))
+    with pytest.raises(bm.BMError) as e:
+        cache.set_left_pad([0, -1])
+    assert e.value.code == 1
+    cache.set_left_pad([3, 0])
+    cache.set_left_pad(None)
+    q, k, v = Inputs(wl, "cuda").block(0, 0, 48)
+    cache.prefill_block(q, k, v, 0, evict_to=wl.K)
+    with pytest.raises(bm.BMError) as e:
+        cache.set_left_pad([1, 1])                                       # only while every cache is empty
+    assert e.value.code == 4
+    cache.close()
+
+
 # ------------------------------------------------------------------ API behaviour on the device
 def test_error_codes_and_state_tracking():
     wl = tiny("errors", dtype="bf16", d=128)
