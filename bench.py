@@ -45,6 +45,8 @@ def parse_args():
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (roofline runs)")
     ap.add_argument("--prompt", type=int, default=None, help="override the workload's prompt length")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
+    ap.add_argument("--ragged", action="store_true",
+                    help="left-padded samples: seeded padding counts in [0, s/2] (sample 0 unpadded); launches eagerly")
     return ap.parse_args()
 
 
@@ -244,8 +246,17 @@ def main():
 
     workspace = torch.empty(max(bm.workspace_bytes(cfg), 256), dtype=torch.uint8, device=dev)
 
+    pads = None
+    if args.ragged:
+        import random
+        rng = random.Random(wl.seed)
+        pads = [0] + [rng.randrange(0, wl.s // 2 + 1) for _ in range(wl.b - 1)]
+        args.no_graph = True     # the padding counts are copied from pageable host memory at the start of a step
+
     def one_step(host_bufs=None, with_decode=True):
         cache = bm.BatchMaxCache(cfg, arena=arena, workspace=workspace)
+        if pads is not None:
+            cache.set_left_pad(pads)
         for layer in range(wl.L):
             for ci, (kind, pos0, I, ev) in enumerate(calls):
                 if kind == "decode" and not with_decode:
@@ -385,7 +396,9 @@ def main():
                 "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
                 "config": cfg_dict(wl, {"parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                                         "prefill_path": "tcgen05" if bm.last_prefill_path() == 1 else "simt-fp32",
-                                        "launch": "eager" if args.no_graph else "one CUDA graph per step, replayed"}),
+                                        "launch": "eager" if args.no_graph else "one CUDA graph per step, replayed",
+                                        "left_pad": "none" if pads is None else
+                                        f"seeded, {sum(pads)} of {wl.b * wl.s} prompt positions are padding"}),
                 "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
                 "clocks": clocks, "prefill_useful_tflop_per_step": 4.0 * wl.d * ppairs / 1e12}
         line.update(extra)
