@@ -104,7 +104,7 @@ class UnitCache:
             # (kv_ids is ascending, so these are the first m entries), minus the padding pairs.
             m = n_old + i + 1
             assert self.kv_ids[m - 1] == pos0 + i
-            vis = np.nonzero(real[:m])[0]
+            vis = slice(0, m) if self.left_pad == 0 else np.nonzero(real[:m])[0]
             for h in range(self.g):
                 logits = self.scale * (self.k[vis] @ q[i, h])
                 w = np.exp(logits - logits.max())
