@@ -47,6 +47,8 @@ struct TcArgs {
   int pos0;
 };
 
+#include "attn_fwd_split.cuh"
+
 // ------------------------------------------------------------------------------------------------------
 // Forward, NT query tiles per CTA.  NT = 2 (large grids): warps 0-3 / 4-7 are the softmax warpgroups of tiles A / B,
 // warp 8 issues the MMAs and owns the tensor memory, warp 9 is the TMA producer; one CTA per SM, both tiles share
@@ -626,8 +628,29 @@ cudaError_t launch_fwd_nt(const CacheView& c, const BlockArgs& a, cudaStream_t s
 // with the other's main loop is worth more than sharing K/V tiles.  BM_FWD_TILES=2 selects the other variant.
 int g_fwd_tiles_override = 0;
 
+template <int D, bool PAD>
+cudaError_t launch_fwd_split(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+  using L = SplitSmem<D>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(attn_fwd_split<D, PAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int R = a.I * c.g;
+  dim3 grid((R + kTileM - 1) / kTileM, c.nsamples * c.Hkv);
+  ProfileScope prof(kAttnFwd, st);
+  attn_fwd_split<D, PAD><<<grid, L::kThreads, L::kTotal, st>>>(g_maps, make_args(c, a));
+  count_launch();
+  return cudaGetLastError();
+}
+
+int g_fwd_kernel = 0;   // 0: two threads per row; 1 / 2: one thread per row, one / two query tiles per CTA (BM_FWD_KERNEL)
+
 template <int D>
 cudaError_t launch_fwd_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+  if (g_fwd_kernel == 0)
+    return c.left_pad != nullptr ? launch_fwd_split<D, true>(c, a, st) : launch_fwd_split<D, false>(c, a, st);
   if (c.left_pad != nullptr)
     return g_fwd_tiles_override == 2 ? launch_fwd_nt<D, 2, true>(c, a, st) : launch_fwd_nt<D, 1, true>(c, a, st);
   return g_fwd_tiles_override == 2 ? launch_fwd_nt<D, 2, false>(c, a, st) : launch_fwd_nt<D, 1, false>(c, a, st);
@@ -671,8 +694,8 @@ bool tc_path_available() {
   static bool init = false;
   if (!init) {
     init = true;
-    const char* e = std::getenv("BM_FWD_TILES");
-    if (e != nullptr) g_fwd_tiles_override = std::atoi(e);
+    const char* e = std::getenv("BM_FWD_KERNEL");   // 0 (default) two threads per row; 1 / 2 one thread per row
+    if (e != nullptr) { g_fwd_kernel = std::atoi(e); g_fwd_tiles_override = g_fwd_kernel; }
   }
   return encode_fn() != nullptr;
 }
