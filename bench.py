@@ -27,7 +27,7 @@ if ROOT not in sys.path:
 METRIC = "P&D evicting-attention tokens/s at max batch; % of TC (prefill) / HBM (decode) peak"
 UNIT = "tokens/s"
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of the same command).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": {"attn_fwd": 91.9e6, "decode": 34.3e6}}   # profiles/attn_fwd_tc_cfg2_traffic.md
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {"cfg2": {"attn_fwd": 92.6e6, "decode": 34.3e6}}   # profiles/attn_fwd_split_cfg2_traffic.md
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -334,7 +334,7 @@ def main():
         achieved = flops_per_step / (attn_ms * 1e-3) / 1e12
         peak = pk["bf16_tflops_sustained"] if wl.dtype == "bf16" else pk["bf16_tflops_sustained"] / 2
         rooflines["attn_fwd"] = {
-            "bound": "tensor", "kernel": "prefill-block attention forward (attn_fwd_tc)", "achieved": achieved,
+            "bound": "tensor", "kernel": "prefill-block attention forward (attn_fwd_split)", "achieved": achieved,
             "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
             "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(wl.name, {}).get("attn_fwd"),
             "peak_source": f"{pk_src} (sustained bf16 matmul)", "launches_per_step": attn_n,
