@@ -224,8 +224,7 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
             p0 = (c0 < nvis && c0 >= nlo) ? p0 : 0.f;
             p1 = (c0 + 1 < nvis && c0 + 1 >= nlo) ? p1 : 0.f;
           }
-          ps0 += p0;
-          ps1 += p1;
+          add2(ps0, ps1, p0, p1);
           pk[e] = pack_bf16(p0, p1);
         }
         tmem_st16(tm_s + lane_addr + c_lo + 16 * ch, pk);

@@ -494,14 +494,14 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
 #pragma unroll
         for (int e = 0; e < 32; e += 2) {
           const int col = cc * 32 + e;
-          float e0 = ex2(fmaf(__uint_as_float(cur[e]), a.scale_log2, -lse_w[col]));
-          float e1 = ex2(fmaf(__uint_as_float(cur[e + 1]), a.scale_log2, -lse_w[col + 1]));
+          float x0, x1;
+          fma2v(x0, x1, __uint_as_float(cur[e]), __uint_as_float(cur[e + 1]), a.scale_log2, -lse_w[col], -lse_w[col + 1]);
+          float e0 = ex2(x0), e1 = ex2(x1);
           if (!nomask) {
             e0 = col >= first_vis ? e0 : 0.f;
             e1 = col + 1 >= first_vis ? e1 : 0.f;
           }
-          p0 += e0;
-          p1 += e1;
+          add2(p0, p1, e0, e1);
         }
         if (cc < 3) {
           tmem_wait_ld();
