@@ -36,6 +36,9 @@ pair) is here as well, :meth:`UnitCache.keep_most_recent` and
 :func:`run_extreme_decoding`, because the library's timed comparison arm is
 checked against it.
 
+Two rules of other methods, as far as Sec. 2 describes them, can replace the
+average (``rule=`` of :class:`UnitCache`): "sum_recent" and "current_query".
+
 Parity unpinned (conventions, not derivable from the paper): the GQA sum, the
 tie direction and the denominator reading above.  Everything else is pinned by
 tests/test_oracle_pins.py.
@@ -52,7 +55,12 @@ class UnitCache:
     Sec. 3.2: ``kv_ids`` (position ids, ascending), ``sum_weights`` and the
     key/value rows themselves."""
 
-    def __init__(self, d: int, g: int = 1, scale: float | None = None, left_pad: int = 0):
+    RULES = ("average", "sum_recent", "current_query")
+
+    def __init__(self, d: int, g: int = 1, scale: float | None = None, left_pad: int = 0,
+                 rule: str = "average"):
+        assert rule in self.RULES
+        self.rule = rule
         self.d = int(d)
         self.g = int(g)
         self.left_pad = int(left_pad)  # positions 0 .. left_pad-1 of this sample are padding (Sec. 3)
@@ -96,6 +104,9 @@ class UnitCache:
         weights = np.zeros((I, self.g, n_old + I)) if return_weights else None
         real = self.kv_ids >= self.left_pad          # padding pairs are masked for every query
         n_real_queries = 0
+        if self.rule == "current_query":
+            # only the weights of the block's last query (its g heads) count, nothing is carried over (Sec. 2)
+            self.sum_weights[:] = 0.0
         for i in range(I):
             if pos0 + i < self.left_pad:
                 continue                             # a padding position: no output, no attention row
@@ -110,7 +121,8 @@ class UnitCache:
                 w = np.exp(logits - logits.max())
                 w = w / w.sum()                      # attn_weights[i] for this head
                 out[i, h] = w @ self.v[vis]
-                self.sum_weights[vis] += w           # sum_weights += attn_weights[i]
+                if self.rule != "current_query" or i == I - 1:
+                    self.sum_weights[vis] += w       # sum_weights += attn_weights[i]
                 if return_weights:
                     weights[i, h, vis] = w
         self.last_pos = pos0 + I - 1
@@ -135,6 +147,23 @@ class UnitCache:
         count = curr_id + 1 - self.kv_ids
         return self.sum_weights / (self.g * count)
 
+    def ranking_scores(self, target: int, curr_id: int | None = None):
+        """The value pairs are ranked by at an eviction down to ``target``.
+        average: ave_weights (Sec. 3.2, the method's rule).
+        sum_recent: the rule Sec. 2 ascribes to H2O -- the cache is split evenly between a window of the most
+          recent pairs and the pairs with the largest sum of past attention weights: the floor(target / 2) most
+          recent pairs rank first (+inf), the others by their raw sum_weights.
+        current_query: the rule Sec. 2 ascribes to TOVA -- the weights of the current query alone (sum_weights
+          holds nothing else under this rule, see process_block)."""
+        if self.rule == "average":
+            return self.ave_weights(curr_id)
+        score = self.sum_weights.copy()
+        if self.rule == "sum_recent":
+            window = int(target) // 2
+            if window > 0:
+                score[len(self) - window:] = np.inf
+        return score
+
     def evict(self, target: int, curr_id: int | None = None, kept_ids=None):
         """Remove the pairs with the smallest ave_weights until ``target`` remain.
 
@@ -148,8 +177,8 @@ class UnitCache:
         target = int(target)
         if target >= n:
             return None
-        ave = self.ave_weights(curr_id)
-        # primary: real pairs before padding pairs (padding always leaves first), then -ave, then id
+        ave = self.ranking_scores(target, curr_id)
+        # primary: real pairs before padding pairs (padding always leaves first), then -score, then id
         order = np.lexsort((self.kv_ids, -ave, self.kv_ids < self.left_pad))
         own_keep = np.sort(order[:target])
         cut = float(ave[order[target - 1]]) if target > 0 else math.inf
@@ -221,7 +250,7 @@ def _trace_entry(unit: UnitCache):
 
 
 def run_north_star(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec: int = 1,
-                   g: int | None = None, scale: float | None = None, left_pad: int = 0):
+                   g: int | None = None, scale: float | None = None, left_pad: int = 0, rule: str = "average"):
     """Blocks of ``block`` prompt tokens (ragged tail allowed), the cache cut back to ``kv_max``
     after every block; then ``steps`` decode steps, cut back to ``kv_max`` whenever the cache
     has grown to ``kv_max + p_dec``.   q: (s+steps, g, d); k, v: (s+steps, d); the first
@@ -229,7 +258,7 @@ def run_north_star(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec: 
     Returns (outputs (s+steps, g, d), trace of kv_ids after every call, unit)."""
     q = np.asarray(q, dtype=np.float64)
     g = q.shape[1] if g is None else g
-    unit = UnitCache(q.shape[2], g, scale, left_pad)
+    unit = UnitCache(q.shape[2], g, scale, left_pad, rule)
     outs, trace = [], []
     pos = 0
     while pos < s:

@@ -569,3 +569,63 @@ def test_left_padding_masked_dense_replay():
                 np.testing.assert_allclose(out[qi, h], sum(wj * v[j] for wj, j in zip(w, js)), atol=1e-12)
         cached = list(trace[call])
         call += 1
+
+
+# ---------------------------------------------------------------- the rules Sec. 2 ascribes to other methods
+def replay_weights(q, k, visible_sets, queries, scale):
+    """weights[(query position, head)] = {key id: softmax weight} recomputed from the original arrays."""
+    out = {}
+    for qi, vis in zip(queries, visible_sets):
+        for h in range(q.shape[1]):
+            lg = np.array([scale * float(q[qi, h] @ k[j]) for j in vis])
+            w = np.exp(lg - lg.max())
+            w /= w.sum()
+            out[(qi, h)] = dict(zip(vis, w))
+    return out
+
+
+@pytest.mark.parametrize("rule", ["current_query", "sum_recent"])
+def test_alternative_rules_against_a_replay_from_the_original_arrays(rule):
+    # every eviction is re-derived from the trace of kept ids and the ORIGINAL q/k arrays: column sums over the
+    # queries that saw a pair (sum_recent) or the last query's weights alone (current_query), never the cache's state
+    s, B, K, steps, g, d = 40, 8, 7, 6, 2, 4
+    q, k, v = rand_qkv(61, s + steps, g, d)
+    out, trace, unit = run_north_star(q, k, v, s, B, K, steps, rule=rule)
+    scale = 1.0 / math.sqrt(d)
+    cached, sums = [], {}
+    calls = [(p0, min(B, s - p0)) for p0 in range(0, s, B)] + [(s + t, 1) for t in range(steps)]
+    for call, (p0, I) in enumerate(calls):
+        cand = list(cached) + list(range(p0, p0 + I))
+        if rule == "current_query":
+            sums = {}
+        for i in range(I):
+            qi = p0 + i
+            vis = list(cached) + list(range(p0, qi + 1))
+            if rule == "current_query" and i != I - 1:
+                continue
+            for (_, h), w in replay_weights(q, k, [vis], [qi], scale).items():
+                for j, wj in w.items():
+                    sums[j] = sums.get(j, 0.0) + wj
+        if len(cand) > K:
+            window = cand[len(cand) - K // 2:] if (rule == "sum_recent" and K // 2 > 0) else []
+            rest = [j for j in cand if j not in window]
+            rest.sort(key=lambda j: (-sums.get(j, 0.0), j))
+            kept = sorted(window + rest[:K - len(window)])
+        else:
+            kept = cand
+        assert kept == list(trace[call]), f"call {call}"
+        sums = {j: sums.get(j, 0.0) for j in kept}
+        cached = kept
+
+
+def test_sum_recent_keeps_its_window_and_current_query_forgets():
+    g, d = 1, 4
+    q, k, v = rand_qkv(67, 30, g, d)
+    u = UnitCache(d, g, rule="sum_recent")
+    u.process_block(q[:20], k[:20], v[:20], 0, evict_to=8)
+    assert set(range(16, 20)) <= set(u.kv_ids.tolist())          # the 4 most recent of 8 always stay
+    u2 = UnitCache(d, g, rule="current_query")
+    _, w = u2.process_block(q[:20], k[:20], v[:20], 0, return_weights=True)
+    np.testing.assert_allclose(u2.sum_weights, w[19, 0], rtol=1e-14)   # the last query's row and nothing else
+    u2.decode_step(q[20], k[20], v[20])
+    assert u2.sum_weights.sum() == pytest.approx(1.0)             # previous sums are gone
