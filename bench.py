@@ -45,6 +45,8 @@ def parse_args():
     ap.add_argument("--batch", type=int, default=None, help="override the workload's batch (roofline runs)")
     ap.add_argument("--prompt", type=int, default=None, help="override the workload's prompt length")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
+    ap.add_argument("--rule", default="average", choices=["average", "sum_recent", "current_query"],
+                    help="eviction rule: the paper's average attention, or one of the two rules of Sec. 2")
     ap.add_argument("--ragged", action="store_true",
                     help="left-padded samples: seeded padding counts in [0, s/2] (sample 0 unpadded); launches eagerly")
     return ap.parse_args()
@@ -228,7 +230,7 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     calls = schedule(wl)
-    cfg = make_config(wl, device=local_rank)
+    cfg = make_config(wl, device=local_rank, rule=args.rule)
     stream = torch.cuda.current_stream()
 
     # ---- inputs resident in HBM (layer 0's stream is reused for every layer: layers are independent)
@@ -397,6 +399,7 @@ def main():
                 "config": cfg_dict(wl, {"parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                                         "prefill_path": "tcgen05" if bm.last_prefill_path() == 1 else "simt-fp32",
                                         "launch": "eager" if args.no_graph else "one CUDA graph per step, replayed",
+                                        "rule": args.rule,
                                         "left_pad": "none" if pads is None else
                                         f"seeded, {sum(pads)} of {wl.b * wl.s} prompt positions are padding"}),
                 "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),

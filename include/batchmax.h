@@ -53,6 +53,17 @@ typedef enum {
 
 typedef enum { BM_F32 = 0, BM_BF16 = 1 } bm_dtype_t;
 
+/* Eviction rule.  BM_RULE_AVERAGE is the method's own (Sec. 3.2).  The other two are the rules Sec. 2 ascribes to
+ * earlier methods, as far as that section describes them, run on the same kernels:
+ *   BM_RULE_SUM_RECENT    (H2O): the cache is split evenly between a window of the most recent pairs and the pairs
+ *                         with the largest sum of past attention weights -- the floor(target / 2) most recent
+ *                         candidates always stay, the others are ranked by their raw sum_weights;
+ *   BM_RULE_CURRENT_QUERY (TOVA): pairs are ranked by the attention weights of the current query alone --
+ *                         sum_weights is overwritten (not accumulated) with the weights of the block's last
+ *                         query, or of the decode step's query, summed over the group's heads.
+ * Ties keep the lower position under every rule. */
+typedef enum { BM_RULE_AVERAGE = 0, BM_RULE_SUM_RECENT = 1, BM_RULE_CURRENT_QUERY = 2 } bm_rule_t;
+
 /* Problem statement: Algorithm 1's inputs (\overline{|kv|}, p) generalised as (K, growth), plus the
  * attention shape.  All sizes in elements. */
 typedef struct {
@@ -68,6 +79,7 @@ typedef struct {
   float softmax_scale;      /* 0 selects 1/sqrt(d)                                            */
   int32_t device;           /* CUDA device ordinal                                            */
   int32_t max_call_samples; /* largest nsamples of any call (sizes the workspace); 0 -> batch */
+  int32_t rule;             /* bm_rule_t: what pairs are ranked by at an eviction; 0 = the paper's  */
 } bm_config_t;
 
 /* ---- cache layout, allocator and memory model (Sec. 1: batch size under a fixed memory budget) ----

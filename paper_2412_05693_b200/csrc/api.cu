@@ -64,6 +64,7 @@ bool config_ok(const bm_config_t* c, bool need_batch) {
   if (!(c->dtype == BM_F32 || c->dtype == BM_BF16)) return false;
   if (!(c->softmax_scale >= 0.f) || std::isinf(c->softmax_scale)) return false;
   if (c->device < 0 || c->max_call_samples < 0) return false;
+  if (c->rule < 0 || c->rule > 2) return false;
   if ((long long)c->kv_max + c->growth > (1 << 24)) return false;
   return true;
 }
@@ -152,6 +153,7 @@ CacheView make_view(const bm_cache* c, int layer, int sample0, int nsamples, int
   v.nsamples = nsamples;
   v.status = c->status;
   v.left_pad = c->has_pad ? c->left_pad + sample0 : nullptr;
+  v.rule = c->cfg.rule;
   return v;
 }
 

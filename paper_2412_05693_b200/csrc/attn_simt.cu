@@ -202,7 +202,9 @@ __global__ void __launch_bounds__(kThreads) score_simt(CacheView c, BlockArgs a)
   for (int row0 = (first_row / kTile) * kTile; row0 < R; row0 += kTile) {
     __syncthreads();
     load_tile<T, D>(sQ, tid, [&](int r) { return query_row_ptr<T, D>(c, a, smp, kh, row0 + r); });
-    if (tid < kTile) sLse[tid] = (row0 + tid < R) ? a.lse[(size_t)unit * R + row0 + tid] : INFINITY;
+    // rule 2 (current query): only the rows of the block's last input contribute
+    if (tid < kTile)
+      sLse[tid] = (row0 + tid < R && (c.rule != 2 || row0 + tid >= R - c.g)) ? a.lse[(size_t)unit * R + row0 + tid] : INFINITY;
     __syncthreads();
     float acc[4][4];
     dot_tile<D>(sQ, sK, ty, tx, acc);
@@ -232,7 +234,10 @@ __global__ void __launch_bounds__(kThreads) score_simt(CacheView c, BlockArgs a)
       const int pad = sample_left_pad(c, smp);
       if (pad > 0 && (j < c.n_old ? c.kv_ids[(size_t)unit * c.cap + j] : a.pos0 + (j - c.n_old)) < pad)
         tot = 0.f;                                  // a padding pair is masked for every query
-      if (j < c.n_old) c.sum_weights[(size_t)unit * c.cap + j] += tot;
+      if (j < c.n_old) {
+        if (c.rule == 2) c.sum_weights[(size_t)unit * c.cap + j] = tot;   // nothing is carried over
+        else c.sum_weights[(size_t)unit * c.cap + j] += tot;
+      }
       else a.new_sum[(size_t)unit * a.I + (j - c.n_old)] = tot;
     }
   }

@@ -45,6 +45,7 @@ struct TcArgs {
   const int* left_pad;
   const int* kv_ids;
   int pos0;
+  int rule;          // 2: only the rows of the block's last input contribute to the column sums, which replace sum_weights
 };
 
 #include "attn_fwd_split.cuh"
@@ -476,7 +477,7 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
       // this tile's log2-sum-exp values; +inf for rows past the block's end (weight 0)
       {
         const int rr = qrow0 + key;
-        sLse[wg * 128 + key] = rr < R ? a.lse2[(size_t)unit * R + rr] : INFINITY;
+        sLse[wg * 128 + key] = (rr < R && (a.rule != 2 || rr >= R - a.g)) ? a.lse2[(size_t)unit * R + rr] : INFINITY;
       }
       named_bar_sync(1 + wg, 128);
       mbar_wait(&bars[C_SFULL + wg], (t / kScoreWG) & 1, abort_flag, a.status);
@@ -526,7 +527,12 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
         const bool in_range = is_old ? j < a.n_old : j < a.I;
         if (pad > 0 && in_range && (is_old ? a.kv_ids[(size_t)unit * a.cap + j] : a.pos0 + j) < pad) tot = 0.f;
       }
-      if (is_old) { if (j < a.n_old) a.sum_weights[(size_t)unit * a.cap + j] += tot; }
+      if (is_old) {
+        if (j < a.n_old) {
+          if (a.rule == 2) a.sum_weights[(size_t)unit * a.cap + j] = tot;   // nothing is carried over
+          else a.sum_weights[(size_t)unit * a.cap + j] += tot;
+        }
+      }
       else if (j < a.I) a.new_sum[(size_t)unit * a.I + j] = tot;
     }
   }
@@ -597,7 +603,7 @@ TcArgs make_args(const CacheView& c, const BlockArgs& a) {
   t.scale_log2 = a.scale * kLog2e;
   t.lse2 = a.lse; t.sum_weights = c.sum_weights; t.new_sum = a.new_sum;
   t.cap = c.cap; t.status = c.status;
-  t.left_pad = c.left_pad; t.kv_ids = c.kv_ids; t.pos0 = a.pos0;
+  t.left_pad = c.left_pad; t.kv_ids = c.kv_ids; t.pos0 = a.pos0; t.rule = c.rule;
   return t;
 }
 

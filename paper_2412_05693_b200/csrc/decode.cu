@@ -196,10 +196,14 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
       s.p[h * n1p + j] = p;
       add += p;
     }
-    const float sw = ((j < c.n_old) ? c.sum_weights[base + j] : 0.f) + add;
+    // rule 2 (current query) keeps this step's weights only
+    const float sw = ((j < c.n_old && c.rule != 2) ? c.sum_weights[base + j] : 0.f) + add;
     s.score[j] = sw;
     if (evict_one) {
-      const float ave = s.id[j] < pad ? -1.f : sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
+      float ave;   // ranking value: average attention (Sec. 3.2), or the raw weights with / without a recent window
+      if (s.id[j] < pad) ave = -1.f;
+      else if (c.rule == 0) ave = sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
+      else ave = (c.rule == 1 && j >= n1 - a.target / 2) ? INFINITY : sw;
       if (ave <= best_ave) { best_ave = ave; best_j = j; }   // j ascends: ties move to the higher position
     } else {
       c.sum_weights[base + j] = sw;

@@ -267,10 +267,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
     } else if (j < c.n_old) {
       old_sw = c.sum_weights[base + j];
     }
-    const float sw = old_sw + add;
+    const float sw = (c.rule == 2 ? 0.f : old_sw) + add;   // rule 2 (current query) keeps this step's weights only
     s.score[j] = sw;
     if (evict_one) {
-      const float ave = s.id[j] < pad ? -1.f : sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
+      float ave;   // ranking value: average attention (Sec. 3.2), or the raw weights with / without a recent window
+      if (s.id[j] < pad) ave = -1.f;
+      else if (c.rule == 0) ave = sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
+      else ave = (c.rule == 1 && j >= n1 - a.target / 2) ? INFINITY : sw;
       if (ave <= best_ave) { best_ave = ave; best_j = j; }   // j ascends: ties move to the higher position
     } else {
       c.sum_weights[base + j] = sw;

@@ -74,7 +74,10 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
   const int pad = sample_left_pad(c, smp);
   auto ave_bits = [&](int j) -> uint32_t {
     const float cnt = (float)(e.curr_id + 1 - s.id[j]);
-    const uint32_t b = __float_as_uint(s.score[j] / (gf * cnt));  // ave >= 0: the bit pattern orders like the value
+    uint32_t b;   // ranking value >= 0: the bit pattern orders like the value
+    if (c.rule == 0) b = __float_as_uint(s.score[j] / (gf * cnt));       // average attention (Sec. 3.2)
+    else if (c.rule == 1 && j >= n_c - target / 2) b = 0x7f800000u;      // window of recent pairs: always kept
+    else b = __float_as_uint(s.score[j]);                                // raw (sum of / current) weights
     if (pad == 0) return b;
     return s.id[j] < pad ? 0u : max(b, 1u);   // padding pairs rank below every real pair (left-padded samples)
   };

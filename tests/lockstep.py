@@ -23,10 +23,10 @@ OUT_TOL = {"bf16": 2e-2, "f32": 1e-4}
 
 
 def make_config(wl: Workload, device: int = 0, growth: int | None = None, batch: int | None = None,
-                max_call_samples: int = 0) -> Config:
+                max_call_samples: int = 0, rule: str = "average") -> Config:
     return Config(batch=wl.b if batch is None else batch, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.d,
                   kv_max=wl.K, block_max=wl.B, growth=max(1, wl.p_dec) if growth is None else growth,
-                  dtype=wl.dtype, n_layers=wl.L, device=device, max_call_samples=max_call_samples)
+                  dtype=wl.dtype, n_layers=wl.L, device=device, max_call_samples=max_call_samples, rule=rule)
 
 
 def _np(t):
@@ -36,7 +36,7 @@ def _np(t):
 def check_kept(unit: UnitCache, gpu_ids: np.ndarray, target: int, stats: dict, where: str):
     """Band check of the GPU's kept set against the oracle's ranking; the oracle then evicts (adopting the
     GPU's set when it differs inside the band)."""
-    ave = unit.ave_weights()
+    ave = unit.ranking_scores(target)             # ave_weights under the paper's rule
     cand = unit.kv_ids
     is_pad = cand < unit.left_pad                 # padding pairs of a left-padded sample rank after every real pair
     order = np.lexsort((cand, -ave, is_pad))
@@ -66,17 +66,17 @@ def check_kept(unit: UnitCache, gpu_ids: np.ndarray, target: int, stats: dict, w
 
 
 def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=None, check_rows_every: int = 8,
-                 growth: int | None = None, sum_rtol: float | None = None, pads=None):
+                 growth: int | None = None, sum_rtol: float | None = None, pads=None, rule: str = "average"):
     """Run `calls` (default: the workload's spec schedule) on the GPU for the whole batch and on the
     oracle for `units` = [(sample, kv_head), ...].  Returns a dict of statistics; raises on any mismatch."""
     dev = torch.device("cuda", device)
     inp = Inputs(wl, dev)
-    cfg = make_config(wl, device, growth)
+    cfg = make_config(wl, device, growth, rule=rule)
     cache = BatchMaxCache(cfg)
     if pads is not None:                            # left-padded samples: pads[sample] padding positions
         cache.set_left_pad(pads)
     g = wl.g
-    oracles = {u: UnitCache(wl.d, g, left_pad=0 if pads is None else pads[u[0]]) for u in units}
+    oracles = {u: UnitCache(wl.d, g, left_pad=0 if pads is None else pads[u[0]], rule=rule) for u in units}
     stats = {"adoptions": 0, "evictions": 0, "max_out_err": 0.0, "max_sum_rel": 0.0, "calls": 0, "tc_calls": 0}
     tol = OUT_TOL[wl.dtype]
     sum_rtol = sum_rtol if sum_rtol is not None else (2e-3 if wl.dtype == "bf16" else 2e-4)

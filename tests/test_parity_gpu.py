@@ -152,6 +152,21 @@ def test_extreme_decoding_arm_on_gpu(dtype, d, kv_bar):
     assert st["calls"] == len(calls)
 
 
+# ------------------------------------------------------------------ the rules of Sec. 2 on the same kernels
+@pytest.mark.parametrize("rule", ["sum_recent", "current_query"])
+@pytest.mark.parametrize("dtype,d,Hq,Hkv", [("bf16", 128, 8, 2), ("f32", 64, 4, 4)])
+def test_alternative_eviction_rules_lockstep(rule, dtype, d, Hq, Hkv):
+    wl = tiny("rules", s=400, B=128, K=96, steps=12, dtype=dtype, d=d, Hq=Hq, Hkv=Hkv)
+    st = run_lockstep(wl, all_units(wl), rule=rule, check_rows_every=2)
+    assert st["evictions"] >= 2 * Hkv * (3 + 12)
+
+
+def test_alternative_rule_with_growth_falls_back_to_the_general_select():
+    # decode evicts 8 pairs at a time: the fused arg-min does not apply, the select kernel ranks by the rule
+    wl = tiny("rules_g", s=256, B=64, K=64, steps=20, p_dec=8, dtype="bf16", d=128, Hq=8, Hkv=2)
+    run_lockstep(wl, all_units(wl), rule="sum_recent", check_rows_every=4)
+
+
 # ------------------------------------------------------------------ left-padded samples (Sec. 3)
 @pytest.mark.parametrize("dtype,d,s,B,K,pads", [
     ("f32", 64, 200, 48, 40, [0, 37, 150]),         # SIMT path; padding inside a block and over whole blocks
