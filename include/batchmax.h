@@ -235,6 +235,15 @@ bm_status_t bm_cache_clear_status(bm_cache_t* cache, void* cuda_stream);
  * normally; bm_cache_status then reports BM_ERR_TIMEOUT and the context stays usable.  Nothing else is touched. */
 bm_status_t bm_selftest_wait_timeout(bm_cache_t* cache, void* cuda_stream);
 
+/* ---- rows moved by compactions (measurement aid: the compaction term of the decode step's memory traffic) ----
+ * While switched on for a handle, every eviction adds the number of cache rows it moves (each row = one key and one
+ * value row read and written) to counters in the arena's status block: the rows behind the first removed pair for
+ * the stable compaction of bm_prefill_block / bm_evict, the rows behind the hole for the one-row shift of an
+ * evicting decode step.  bm_cache_moved_rows returns the total so far (and clears it when reset != 0); it
+ * synchronises cuda_stream. */
+bm_status_t bm_cache_count_moved_rows(bm_cache_t* cache, int32_t on);
+bm_status_t bm_cache_moved_rows(bm_cache_t* cache, uint64_t* rows /*HOST out*/, int32_t reset, void* cuda_stream);
+
 /* ---- per-kernel timing (measurement aid; the paper has no counterpart) ----
  * While enabled, every kernel launch of this library is bracketed by two CUDA events on its stream.
  * bm_profile_read waits for the recorded launches of one kernel class, returns their summed duration in

@@ -50,6 +50,8 @@ SIGNATURES = {
     "bm_evict": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp]),
     "bm_keep_most_recent": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp]),
     "bm_cache_set_left_pad": (_i32, [_vp, _vp, _vp]),
+    "bm_cache_count_moved_rows": (_i32, [_vp, _i32]),
+    "bm_cache_moved_rows": (_i32, [_vp, C.POINTER(C.c_uint64), _i32, _vp]),
     "bm_staging_bytes": (_i32, [_cfgp, _i32, _i32, C.POINTER(_sz)]),
     "bm_prefill_block_host": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _i32, _i32, _vp, _i32, _vp, _sz, _vp]),
     "bm_decode_step_host": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp, _sz, _vp]),
@@ -273,6 +275,14 @@ class BatchMaxCache:
         arr = (C.c_int32 * len(pads))(*pads)
         _check(lib().bm_cache_set_left_pad(self.h, C.cast(arr, C.c_void_p), _stream(stream)),
                "bm_cache_set_left_pad")
+
+    def count_moved_rows(self, on: bool = True):
+        _check(lib().bm_cache_count_moved_rows(self.h, 1 if on else 0), "bm_cache_count_moved_rows")
+
+    def moved_rows(self, reset: bool = False, stream=None) -> int:
+        out = C.c_uint64(0)
+        _check(lib().bm_cache_moved_rows(self.h, C.byref(out), 1 if reset else 0, _stream(stream)), "bm_cache_moved_rows")
+        return int(out.value)
 
     # -- host-fed variants ---------------------------------------------------------------------------
     def _stage(self, ns, I):

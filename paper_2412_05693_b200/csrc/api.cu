@@ -100,6 +100,7 @@ struct bm_cache {
   float* ws_new_sum;
   int32_t* left_pad = nullptr;   // [batch] device copy of the samples' padding counts (in the workspace)
   bool has_pad = false;          // some sample is left-padded
+  bool count_moves = false;      // compactions add the rows they move to the counters in the status block
   std::vector<int32_t> n, curr_id;  // [L * b] host mirror
   // host-fed calls run as a three-stage pipeline on streams owned by the handle -- input copies, the pass,
   // the output copy -- so that the three stages of consecutive calls overlap (PCIe is full duplex); the
@@ -154,6 +155,7 @@ CacheView make_view(const bm_cache* c, int layer, int sample0, int nsamples, int
   v.status = c->status;
   v.left_pad = c->has_pad ? c->left_pad + sample0 : nullptr;
   v.rule = c->cfg.rule;
+  v.moved = c->count_moves ? reinterpret_cast<unsigned long long*>(c->status + 16) : nullptr;
   return v;
 }
 
@@ -512,6 +514,28 @@ bm_status_t bm_cache_set_left_pad(bm_cache_t* c, const int32_t* pads, void* cuda
   if (cudaMemcpyAsync(c->left_pad, pads, sizeof(int32_t) * (size_t)c->cfg.batch, cudaMemcpyHostToDevice,
                       static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
     return BM_ERR_CUDA;
+  return BM_OK;
+}
+
+bm_status_t bm_cache_count_moved_rows(bm_cache_t* c, int32_t on) {
+  if (c == nullptr) return BM_ERR_INVALID;
+  c->count_moves = on != 0;
+  return BM_OK;
+}
+
+bm_status_t bm_cache_moved_rows(bm_cache_t* c, uint64_t* rows, int32_t reset, void* cuda_stream) {
+  if (c == nullptr || rows == nullptr) return BM_ERR_INVALID;
+  bm_status_t s = set_device(c);
+  if (s != BM_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned long long part[16];
+  void* dev = c->status + 16;
+  if (cudaMemcpyAsync(part, dev, sizeof(part), cudaMemcpyDeviceToHost, st) != cudaSuccess) return BM_ERR_CUDA;
+  if (reset && cudaMemsetAsync(dev, 0, sizeof(part), st) != cudaSuccess) return BM_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return BM_ERR_CUDA;
+  uint64_t tot = 0;
+  for (unsigned long long v : part) tot += v;
+  *rows = tot;
   return BM_OK;
 }
 

@@ -19,6 +19,7 @@ struct CacheView {
   int32_t nsamples;
   int32_t* status;     // device status word
   const int32_t* left_pad;  // [nsamples] padding positions at the start of each sample of the range, or null
+  unsigned long long* moved;  // [16] counters of rows moved by compactions (unit & 15), or null when not counting
   int32_t rule;             // 0 average attention (Sec. 3.2), 1 sum + window of recent pairs, 2 current query (Sec. 2)
 };
 

@@ -228,6 +228,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
       if (oa < best_ave || (oa == best_ave && oj > best_j)) { best_ave = oa; best_j = oj; }
     }
     hole = best_j;
+    if (c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)(n1 - 1 - hole));
     // sum_weights / kv_ids in their final places: rows behind the hole move up by one
     for (int j = tid; j < n1; j += kDecThreads) {
       if (j < hole) { if (j >= 0) c.sum_weights[base + j] = s.score[j]; }

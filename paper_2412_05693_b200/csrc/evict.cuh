@@ -164,6 +164,8 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
   }
   __syncthreads();
   const int first_moved = s.misc[2];
+  if (c.moved != nullptr && tid == 0 && first_moved < target)   // stable compaction: every row from there on moves
+    atomicAdd(&c.moved[unit & 15], (unsigned long long)(target - first_moved));
 
   for (int r = first_moved + tid; r < target; r += NT) {
     const int j = s.src[r];

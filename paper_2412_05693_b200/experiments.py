@@ -146,8 +146,10 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
         arena = torch.empty(need, dtype=torch.uint8, device=dev)
     assert arena.numel() >= need, "arena smaller than the memory model asks for"
     cache = BatchMaxCache(cfg, arena=arena[:need])
+    cache.count_moved_rows(True)
     inp = Inputs(wl, dev)
     t_pre, t_dec = Timer(), Timer()
+    moved_pre = None
     ms_pre = ms_dec = 0.0
     layers = range(wl.L) if layers is None else layers
     out_blk = torch.empty(micro, cfg.block_max, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
@@ -158,6 +160,8 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
     for layer in layers:
         n, in_decode, pending = 0, False, 0
         for kind, pos0, I, arg in calls:
+            if kind == "decode" and not in_decode:
+                moved_pre = cache.moved_rows(reset=True)
             in_decode = in_decode or kind == "decode"
             timer = t_dec if in_decode else t_pre
             if kind == "prefill":
@@ -169,11 +173,17 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
                 pairs += I * n + I * (I + 1) // 2
                 n = n + I if arg < 0 else min(n + I, arg)
             elif kind == "decode":
-                for s0 in range(0, batch, micro_dec):
-                    ns = min(micro_dec, batch - s0)
-                    q, k, v = inp.block(layer, pos0, 1, s0, ns)
-                    q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
-                    timer(lambda: cache.decode_step(q, k, v, out=out_dec[:ns], evict_to=arg, layer=layer, sample0=s0))
+                # one token per sample is small: the step's inputs are drawn for the whole batch first, then the calls
+                # of all sample ranges run back to back inside one timed region
+                q, k, v = inp.block(layer, pos0, 1)
+                q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
+
+                def step_calls():
+                    for s0 in range(0, batch, micro_dec):
+                        ns = min(micro_dec, batch - s0)
+                        cache.decode_step(q[s0:s0 + ns], k[s0:s0 + ns], v[s0:s0 + ns], out=out_dec[:ns], evict_to=arg,
+                                          layer=layer, sample0=s0)
+                timer(step_calls)
                 dec_rows += n + 1
                 n = n + 1 if arg < 0 else min(n + 1, arg)
             else:
@@ -191,6 +201,9 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
         ms_pre += t_pre.total_ms()
         ms_dec += t_dec.total_ms()
     assert cache.status() == 0
+    moved_dec = cache.moved_rows(reset=True)
+    if moved_pre is None:
+        moved_pre, moved_dec = moved_dec, 0
     n_layers = len(list(layers))
     n_end, cur = cache.length(layer=list(layers)[-1], sample=batch - 1)
     assert n_end == n, "host mirror disagrees with the schedule's own count"
@@ -212,10 +225,15 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
         "prefill_frac_of_peak": flops / (ms_pre * 1e-3) / 1e12 / tf,
         "decode_gbs": dec_bytes / (ms_dec * 1e-3) / 1e9 if ms_dec > 0 else None,
         "decode_frac_of_peak": dec_bytes / (ms_dec * 1e-3) / 1e9 / hbm if ms_dec > 0 else None,
+        "decode_rows_moved": moved_dec, "prefill_rows_moved": moved_pre,
+        "decode_gbs_with_moves": (dec_bytes + moved_dec * 2.0 * wl.d * e) / (ms_dec * 1e-3) / 1e9 if ms_dec > 0 else None,
+        "decode_frac_with_moves": (dec_bytes + moved_dec * 2.0 * wl.d * e) / (ms_dec * 1e-3) / 1e9 / hbm
+        if ms_dec > 0 else None,
         "peaks": {"hbm_gbs": hbm, "bf16_tflops_sustained": tf, "source": src},
         "note": "prefill = every call before the first decode step (attention, score pass, evictions; the whole call, "
                 "not the forward kernel alone); decode = every call from the first decode step on; decode bytes "
-                "exclude compaction moves; every call timed with its own CUDA events",
+                "exclude compaction moves; every prefill call and every decode step (all its sample ranges) timed with its own "
+                "CUDA events",
     }
     if arm in ("alg1", "ed"):
         res["kv_bar"] = kv_bar

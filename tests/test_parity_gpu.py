@@ -207,6 +207,36 @@ def test_left_pad_setter_errors():
     cache.close()
 
 
+def test_moved_row_counters_match_the_kept_sets():
+    # rows a compaction moves = rows from the first one whose content changes to the end of the kept set
+    wl = tiny("moved", b=2, s=192, B=64, K=40, steps=10, dtype="bf16", d=128, Hq=8, Hkv=2)
+    cache = bm.BatchMaxCache(make_config(wl))
+    cache.count_moved_rows(True)
+    inp = Inputs(wl, "cuda")
+    units = all_units(wl)
+    before = {u: [] for u in units}
+    expected = 0
+    for kind, pos0, I, ev in schedule(wl):
+        q, k, v = inp.block(0, pos0, I)
+        if kind == "prefill":
+            cache.prefill_block(q, k, v, pos0, evict_to=ev)
+        else:
+            cache.decode_step(q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous(), evict_to=ev)
+        for u in units:
+            ids = cache.export(0, u[0], u[1])[0].tolist()
+            n_old = len(before[u])
+            cand = before[u] + list(range(pos0, pos0 + I))
+            evicted = len(ids) < len(cand)
+            if kind == "prefill" or evicted:      # a decode step that only appends moves nothing
+                first = next((r for r in range(len(ids)) if ids[r] != cand[r] or r >= n_old), len(ids))
+                expected += len(ids) - first
+            before[u] = ids
+    assert cache.moved_rows() == expected
+    assert cache.moved_rows(reset=True) == expected
+    assert cache.moved_rows() == 0
+    cache.close()
+
+
 # ------------------------------------------------------------------ API behaviour on the device
 def test_error_codes_and_state_tracking():
     wl = tiny("errors", dtype="bf16", d=128)
