@@ -255,14 +255,18 @@ def main():
         pads = [0] + [rng.randrange(0, wl.s // 2 + 1) for _ in range(wl.b - 1)]
         args.no_graph = True     # the padding counts are copied from pageable host memory at the start of a step
 
-    def one_step(host_bufs=None, with_decode=True):
+    def one_step(host_bufs=None, with_decode=True, moved=None):
         cache = bm.BatchMaxCache(cfg, arena=arena, workspace=workspace)
         if pads is not None:
             cache.set_left_pad(pads)
+        if moved is not None:                 # count the rows the compactions move, prefill and decode apart
+            cache.count_moved_rows(True)
         for layer in range(wl.L):
             for ci, (kind, pos0, I, ev) in enumerate(calls):
                 if kind == "decode" and not with_decode:
                     continue
+                if moved is not None and kind == "decode" and (ci == 0 or calls[ci - 1][0] != "decode"):
+                    moved["prefill"] = moved.get("prefill", 0) + cache.moved_rows(reset=True)
                 if host_bufs is None:
                     q, k, v = dev_in[ci]
                     if kind == "prefill":
@@ -275,6 +279,8 @@ def main():
                         cache.prefill_block_host(q, k, v, pos0, o, evict_to=ev, layer=layer)
                     else:
                         cache.decode_step_host(q, k, v, o, evict_to=ev, layer=layer)
+            if moved is not None:
+                moved["decode"] = moved.get("decode", 0) + cache.moved_rows(reset=True)
         return cache
 
     def timed(n_warm, n_steps, host_bufs=None, use_graph=False, with_decode=True):
@@ -354,10 +360,15 @@ def main():
         in_region_ms = max(ms_step - ms_prefill_only, 1e-6) * wl.L if not args.no_graph else dec_ms
         gbs_events = gbs
         gbs = dec_bytes / (in_region_ms * 1e-3) / 1e9
+        moved = {}
+        one_step(moved=moved).close()             # one more eager pass with the device-side counters on
+        move_bytes = moved.get("decode", 0) * 2.0 * wl.d * e
         rooflines["decode"] = {
             "bound": "hbm", "kernel": "decode step with score update and eviction (decode_mma_kernel)",
             "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": gbs / pk["hbm_gbs"],
             "achieved_with_per_launch_events": gbs_events, "ms_in_timed_region": in_region_ms,
+            "achieved_with_compaction_writes": (dec_bytes + move_bytes) / (in_region_ms * 1e-3) / 1e9,
+            "rows_moved_per_cache_and_step": moved.get("decode", 0) / max(1, wl.b * wl.Hkv * dec_n),
             "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(wl.name, {}).get("decode"),
             "peak_source": f"{pk_src} (HBM copy)", "launches_per_step": dec_n,
             "avg_launch_ms": dec_ms / max(dec_n, 1),
