@@ -246,12 +246,8 @@ __global__ void __launch_bounds__(kThreads) score_simt(CacheView c, BlockArgs a)
 template <typename T, int D>
 cudaError_t launch_attn_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
   const size_t smem = sizeof(float) * (2 * kTile * (D + 1) + kTile * (kTile + 1) + 4 * kTile);
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = configured.ensure(attn_fwd_simt<T, D>, (size_t)(smem)); e != cudaSuccess) return e;
   const int R = a.I * c.g;
   dim3 grid((R + kTile - 1) / kTile, c.nsamples * c.Hkv);
   ProfileScope prof(kAttnFwd, st);
@@ -263,12 +259,8 @@ cudaError_t launch_attn_t(const CacheView& c, const BlockArgs& a, cudaStream_t s
 template <typename T, int D>
 cudaError_t launch_score_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
   const size_t smem = sizeof(float) * (2 * kTile * (D + 1) + 16 * kTile + kTile);
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(score_simt<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = configured.ensure(score_simt<T, D>, (size_t)(smem)); e != cudaSuccess) return e;
   dim3 grid((c.n_old + a.I + kTile - 1) / kTile, c.nsamples * c.Hkv);
   ProfileScope prof(kScore, st);
   score_simt<T, D><<<grid, kThreads, smem, st>>>(c, a);

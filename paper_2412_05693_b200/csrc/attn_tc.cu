@@ -608,19 +608,14 @@ TcArgs make_args(const CacheView& c, const BlockArgs& a) {
 }
 
 // maps of the call in flight: built by the forward launcher, reused by the score launcher
-TcMaps g_maps;
-const void* g_maps_q = nullptr;
+thread_local TcMaps g_maps;            // per thread: handles used from different threads do not share them
+thread_local const void* g_maps_q = nullptr;
 
 template <int D, int NT, bool PAD>
 cudaError_t launch_fwd_nt(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
   using L = FwdSmem<D, NT>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_tc<D, NT, PAD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         L::kTotal);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = configured.ensure(attn_fwd_tc<D, NT, PAD>, (size_t)(L::kTotal)); e != cudaSuccess) return e;
   const int R = a.I * c.g;
   dim3 grid((R + NT * kTileM - 1) / (NT * kTileM), c.nsamples * c.Hkv);
   ProfileScope prof(kAttnFwd, st);
@@ -637,12 +632,8 @@ int g_fwd_tiles_override = 0;
 template <int D, bool PAD>
 cudaError_t launch_fwd_split(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
   using L = SplitSmem<D>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_split<D, PAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = configured.ensure(attn_fwd_split<D, PAD>, (size_t)(L::kTotal)); e != cudaSuccess) return e;
   const int R = a.I * c.g;
   dim3 grid((R + kTileM - 1) / kTileM, c.nsamples * c.Hkv);
   ProfileScope prof(kAttnFwd, st);
@@ -664,12 +655,8 @@ cudaError_t launch_fwd_t(const CacheView& c, const BlockArgs& a, cudaStream_t st
 
 template <int D>
 cudaError_t launch_score_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(score_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScoreSmem<D>::kTotal);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t e = configured.ensure(score_tc<D>, (size_t)(ScoreSmem<D>::kTotal)); e != cudaSuccess) return e;
   const int t_old = (c.n_old + kTileN - 1) / kTileN, t_new = (a.I + kTileN - 1) / kTileN;
   dim3 grid(t_old + t_new, c.nsamples * c.Hkv);
   ProfileScope prof(kScore, st);

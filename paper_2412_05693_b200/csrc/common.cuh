@@ -69,6 +69,25 @@ cudaError_t launch_wait_timeout_selftest(int* status, cudaStream_t st);
 cudaError_t launch_attn_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used);
 cudaError_t launch_score_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used);
 
+// cudaFuncSetAttribute applies to the current device only, so the largest dynamic shared-memory size a kernel has
+// been configured for is remembered per device (a process may hold handles on several GPUs).
+struct SmemConfigured {
+  size_t bytes[64] = {};
+  template <typename Kernel>
+  cudaError_t ensure(Kernel kernel, size_t smem) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (smem > bytes[dev]) {
+      e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      bytes[dev] = smem;
+    }
+    return cudaSuccess;
+  }
+};
+
 extern unsigned long long g_launch_count;
 inline void count_launch(int n = 1) { g_launch_count += (unsigned long long)n; }
 

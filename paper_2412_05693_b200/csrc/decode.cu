@@ -333,12 +333,8 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
 template <typename T, int D, int G>
 cudaError_t launch_t(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
   const size_t smem = decode_smem_bytes(D, G, c.n_old + 1, a.target);
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t err = cudaFuncSetAttribute(decode_kernel<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (err != cudaSuccess) return err;
-    configured = smem;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t err = configured.ensure(decode_kernel<T, D, G>, smem); err != cudaSuccess) return err;
   ProfileScope prof(kDecode, st);
   decode_kernel<T, D, G><<<c.nsamples * c.Hkv, kDecThreads, smem, st>>>(c, a);
   count_launch();

@@ -416,12 +416,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
 template <int D, int G>
 cudaError_t launch_t(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
   const size_t smem = decode_mma_smem_bytes(D, G, c.n_old + 1, a.target);
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t err = cudaFuncSetAttribute(decode_mma_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (err != cudaSuccess) return err;
-    configured = smem;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t err = configured.ensure(decode_mma_kernel<D, G>, smem); err != cudaSuccess) return err;
   ProfileScope prof(kDecode, st);
   decode_mma_kernel<D, G><<<c.nsamples * c.Hkv, kThreads, smem, st>>>(c, a);
   count_launch();

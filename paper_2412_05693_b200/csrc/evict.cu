@@ -17,12 +17,8 @@ __global__ void __launch_bounds__(kEvictThreads) evict_kernel(CacheView c, Evict
 template <typename T, int D>
 cudaError_t launch_t(const CacheView& c, const EvictArgs& e, cudaStream_t st) {
   const size_t smem = evict_smem_bytes(c.n_old + e.I, e.target);
-  static size_t configured = 0;
-  if (smem > configured) {
-    cudaError_t err = cudaFuncSetAttribute(evict_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (err != cudaSuccess) return err;
-    configured = smem;
-  }
+  static SmemConfigured configured;
+  if (cudaError_t err = configured.ensure(evict_kernel<T, D>, smem); err != cudaSuccess) return err;
   ProfileScope prof(kEvict, st);
   evict_kernel<T, D><<<c.nsamples * c.Hkv, kEvictThreads, smem, st>>>(c, e);
   count_launch();
