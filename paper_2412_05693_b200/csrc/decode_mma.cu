@@ -12,9 +12,12 @@
 namespace bm {
 namespace {
 
-constexpr int kThreads = 256;   // two CTAs per SM measured faster than one CTA of 512 threads at every batch size
-constexpr int kWarps = kThreads / 32;
-constexpr int kRowsPerIter = kWarps * 16;   // one 16-key tile per warp and iteration
+// CTA size NT (template parameter): 256 threads, two CTAs per SM, when the grid is at most about two CTAs per SM --
+// a step's time is then one CTA's latency, and eight warps finish a cache sooner; 128 threads, four CTAs per SM,
+// for larger grids -- four independent caches per SM keep the memory pipe busy while others sit in their
+// softmax / arg-min / reduction phases (0.85 against 0.71 of the HBM copy peak at 16384 caches of 512 pairs; one CTA
+// of 512 threads per SM measured worst at every size).
+constexpr int kMaxWarps = 8;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct DecodeArgs {
@@ -36,7 +39,7 @@ struct Smem {
   float* ored;    // [warps][G][D]
 };
 
-__host__ __device__ inline size_t smem_layout(unsigned char* base, int d, int g, int n1, Smem* s) {
+__host__ __device__ inline size_t smem_layout(unsigned char* base, int d, int g, int n1, int kWarps, Smem* s) {
   const size_t n1t = (size_t)((n1 + 15) & ~15);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) & ~size_t(15); return o; };
@@ -79,16 +82,18 @@ __device__ __forceinline__ uint4 ldg16_or_zero(const __nv_bfloat16* p, bool ok) 
   return ok ? ld_global_16(p) : make_uint4(0u, 0u, 0u, 0u);
 }
 
-template <int D, int G>
-__global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, DecodeArgs a) {
+template <int D, int G, int NT>
+__global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, DecodeArgs a) {
   using T = __nv_bfloat16;
+  constexpr int kThreads = NT, kWarps = NT / 32;
+  constexpr int kRowsPerIter = kWarps * 16;   // one 16-key tile per warp and iteration
   constexpr int QR = D / 32;   // 32-element rounds of the logits contraction
   constexpr int VR = D / 64;   // 64-element rounds of the output contraction
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int n1 = c.n_old + 1;
   const int n1t = (n1 + 15) & ~15;
   Smem s;
-  smem_layout(smem_raw, D, G, n1, &s);
+  smem_layout(smem_raw, D, G, n1, kWarps, &s);
 
   const int unit = blockIdx.x, smp = unit / c.Hkv, kh = unit % c.Hkv;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -413,15 +418,29 @@ __global__ void __launch_bounds__(kThreads, 2) decode_mma_kernel(CacheView c, De
   }
 }
 
-template <int D, int G>
-cudaError_t launch_t(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
-  const size_t smem = decode_mma_smem_bytes(D, G, c.n_old + 1, a.target);
+template <int D, int G, int NT>
+cudaError_t launch_nt(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
+  const size_t smem = decode_mma_smem_bytes(D, G, c.n_old + 1, a.target);   // sized for the larger CTA
   static SmemConfigured configured;
-  if (cudaError_t err = configured.ensure(decode_mma_kernel<D, G>, smem); err != cudaSuccess) return err;
+  if (cudaError_t err = configured.ensure(decode_mma_kernel<D, G, NT>, smem); err != cudaSuccess) return err;
   ProfileScope prof(kDecode, st);
-  decode_mma_kernel<D, G><<<c.nsamples * c.Hkv, kThreads, smem, st>>>(c, a);
+  decode_mma_kernel<D, G, NT><<<c.nsamples * c.Hkv, NT, smem, st>>>(c, a);
   count_launch();
   return cudaGetLastError();
+}
+
+int sm_count() {   // of the current device
+  static int count[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (count[dev] == 0 && cudaDeviceGetAttribute(&count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    count[dev] = 148;
+  return count[dev];
+}
+
+template <int D, int G>
+cudaError_t launch_t(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
+  return c.nsamples * c.Hkv > 2 * sm_count() ? launch_nt<D, G, 128>(c, a, st) : launch_nt<D, G, 256>(c, a, st);
 }
 
 template <int D>
@@ -438,7 +457,7 @@ cudaError_t launch_g(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
 }  // namespace
 
 size_t decode_mma_smem_bytes(int d, int g, int n_rows, int target) {
-  const size_t attn = smem_layout(nullptr, d, g, n_rows, nullptr);
+  const size_t attn = smem_layout(nullptr, d, g, n_rows, kMaxWarps, nullptr);
   const size_t ev = (target >= 0 && target < n_rows - 1) ? evict_smem_bytes(n_rows, target) : 0;
   return attn > ev ? attn : ev;
 }
