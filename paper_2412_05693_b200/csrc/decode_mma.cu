@@ -7,6 +7,8 @@
 // Both contractions are invariant under a permutation of the contracted index, and the output index of the
 // second one can be un-permuted when it is written, so every thread loads whole 16-byte pieces of cache
 // rows (coalesced) and the MMA fragment slots are assigned to whatever elements those loads delivered.
+#include <cstdlib>
+
 #include "evict.cuh"
 
 namespace bm {
@@ -15,8 +17,10 @@ namespace {
 // CTA size NT (template parameter): 256 threads, two CTAs per SM, when the grid is at most about two CTAs per SM --
 // a step's time is then one CTA's latency, and eight warps finish a cache sooner; 128 threads, four CTAs per SM,
 // for larger grids -- four independent caches per SM keep the memory pipe busy while others sit in their
-// softmax / arg-min / reduction phases (0.85 against 0.71 of the HBM copy peak at 16384 caches of 512 pairs; one CTA
-// of 512 threads per SM measured worst at every size).
+// softmax / arg-min / reduction phases (0.85 against 0.71 of the HBM copy peak at 16384 caches of 512 pairs) -- as
+// long as four of them fit into shared memory, which grows with the cache length; beyond that the larger CTA is
+// faster again (0.84 against 0.65 at 2048 caches of 2048 pairs).  One CTA of 512 threads per SM measured worst at
+// every size.
 constexpr int kMaxWarps = 8;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -438,9 +442,24 @@ int sm_count() {   // of the current device
   return count[dev];
 }
 
+int forced_threads() {   // BM_DECODE_THREADS=128|256 overrides the choice below (tuning aid)
+  static int v = -1;
+  if (v < 0) {
+    const char* e = std::getenv("BM_DECODE_THREADS");
+    v = e != nullptr ? std::atoi(e) : 0;
+  }
+  return v;
+}
+
 template <int D, int G>
 cudaError_t launch_t(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
-  return c.nsamples * c.Hkv > 2 * sm_count() ? launch_nt<D, G, 128>(c, a, st) : launch_nt<D, G, 256>(c, a, st);
+  const int f = forced_threads();
+  // four small CTAs per SM only pay for short caches: all four must fit into shared memory (up to about 1500 pairs
+  // at g = 4), and beyond that length the larger CTA measured faster at every group size (g = 1, 4096 pairs, 2000
+  // caches: 0.96 against 0.69)
+  const bool four_fit = c.n_old + 1 <= 1536 && smem_layout(nullptr, D, G, c.n_old + 1, 4, nullptr) <= 56 * 1024;
+  const bool small_ctas = f == 128 || (f != 256 && four_fit && c.nsamples * c.Hkv > 2 * sm_count());
+  return small_ctas ? launch_nt<D, G, 128>(c, a, st) : launch_nt<D, G, 256>(c, a, st);
 }
 
 template <int D>
