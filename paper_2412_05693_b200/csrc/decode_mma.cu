@@ -86,7 +86,9 @@ __device__ __forceinline__ uint4 ldg16_or_zero(const __nv_bfloat16* p, bool ok) 
   return ok ? ld_global_16(p) : make_uint4(0u, 0u, 0u, 0u);
 }
 
-template <int D, int G, int NT>
+// PLAIN: no left padding, the paper's own eviction rule, no counting of moved rows -- the instance the common case
+// runs, free of those branches.
+template <int D, int G, int NT, bool PLAIN>
 __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, DecodeArgs a) {
   using T = __nv_bfloat16;
   constexpr int kThreads = NT, kWarps = NT / 32;
@@ -198,9 +200,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
   // and across warps through shared memory in a fixed order.
   // left-padded sample: padding pairs are masked and leave first (each thread masks the rows whose ids it
   // loaded itself); a query at a padding position, which no real decode step is, gets zero output and no weights
-  const int pad = sample_left_pad(c, smp);
-  const bool q_real = a.pos >= pad;
-  if (pad > 0 && q_real) {
+  const int pad = PLAIN ? 0 : sample_left_pad(c, smp);
+  const int rule = PLAIN ? 0 : c.rule;
+  const bool q_real = PLAIN || a.pos >= pad;
+  if (!PLAIN && pad > 0 && q_real) {
     for (int j = tid; j < n1; j += kThreads)
       if (s.id[j] < pad) {
 #pragma unroll
@@ -276,13 +279,13 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
     } else if (j < c.n_old) {
       old_sw = c.sum_weights[base + j];
     }
-    const float sw = (c.rule == 2 ? 0.f : old_sw) + add;   // rule 2 (current query) keeps this step's weights only
+    const float sw = (rule == 2 ? 0.f : old_sw) + add;   // rule 2 (current query) keeps this step's weights only
     s.score[j] = sw;
     if (evict_one) {
       float ave;   // ranking value: average attention (Sec. 3.2), or the raw weights with / without a recent window
-      if (s.id[j] < pad) ave = -1.f;
-      else if (c.rule == 0) ave = sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
-      else ave = (c.rule == 1 && j >= n1 - a.target / 2) ? INFINITY : sw;
+      if (!PLAIN && s.id[j] < pad) ave = -1.f;
+      else if (rule == 0) ave = sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
+      else ave = (rule == 1 && j >= n1 - a.target / 2) ? INFINITY : sw;
       if (ave <= best_ave) { best_ave = ave; best_j = j; }   // j ascends: ties move to the higher position
     } else {
       c.sum_weights[base + j] = sw;
@@ -307,7 +310,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
       if (oa < best_ave || (oa == best_ave && oj > best_j)) { best_ave = oa; best_j = oj; }
     }
     hole = best_j;
-    if (c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)(n1 - 1 - hole));
+    if (!PLAIN && c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)(n1 - 1 - hole));
     // sum_weights / kv_ids in their final places: rows behind the hole move up by one
     for (int j = tid; j < n1; j += kThreads) {
       if (j < hole) c.sum_weights[base + j] = s.score[j];
@@ -422,15 +425,21 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
   }
 }
 
-template <int D, int G, int NT>
-cudaError_t launch_nt(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
+template <int D, int G, int NT, bool PLAIN>
+cudaError_t launch_nt_p(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
   const size_t smem = decode_mma_smem_bytes(D, G, c.n_old + 1, a.target);   // sized for the larger CTA
   static SmemConfigured configured;
-  if (cudaError_t err = configured.ensure(decode_mma_kernel<D, G, NT>, smem); err != cudaSuccess) return err;
+  if (cudaError_t err = configured.ensure(decode_mma_kernel<D, G, NT, PLAIN>, smem); err != cudaSuccess) return err;
   ProfileScope prof(kDecode, st);
-  decode_mma_kernel<D, G, NT><<<c.nsamples * c.Hkv, NT, smem, st>>>(c, a);
+  decode_mma_kernel<D, G, NT, PLAIN><<<c.nsamples * c.Hkv, NT, smem, st>>>(c, a);
   count_launch();
   return cudaGetLastError();
+}
+
+template <int D, int G, int NT>
+cudaError_t launch_nt(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
+  const bool plain = c.left_pad == nullptr && c.rule == 0 && c.moved == nullptr;
+  return plain ? launch_nt_p<D, G, NT, true>(c, a, st) : launch_nt_p<D, G, NT, false>(c, a, st);
 }
 
 int sm_count() {   // of the current device
