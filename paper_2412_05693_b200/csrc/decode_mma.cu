@@ -284,7 +284,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
     if (evict_one) {
       float ave;   // ranking value: average attention (Sec. 3.2), or the raw weights with / without a recent window
       if (!PLAIN && s.id[j] < pad) ave = -1.f;
-      else if (rule == 0) ave = sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
+      // fast division: the IEEE routine takes a slow path for the tiny sums of long-evicted histories (4 % of the step)
+      else if (rule == 0) ave = __fdividef(sw, (float)G * (float)(a.pos + 1 - s.id[j]));
       else ave = (rule == 1 && j >= n1 - a.target / 2) ? INFINITY : sw;
       if (ave <= best_ave) { best_ave = ave; best_j = j; }   // j ascends: ties move to the higher position
     } else {
