@@ -85,6 +85,16 @@ __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1
 __device__ __forceinline__ uint4 ldg16_or_zero(const __nv_bfloat16* p, bool ok) {
   return ok ? ld_global_16(p) : make_uint4(0u, 0u, 0u, 0u);
 }
+// 32 bytes (16 elements) with one 256-bit load: the four lanes that share a key row then cover a whole 128-byte
+// line per request instead of half of one
+__device__ __forceinline__ void ldg32_or_zero(const __nv_bfloat16* p, bool ok, uint4& lo, uint4& hi) {
+  lo = make_uint4(0u, 0u, 0u, 0u);
+  hi = lo;
+  if (ok)
+    asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(lo.x), "=r"(lo.y), "=r"(lo.z), "=r"(lo.w), "=r"(hi.x), "=r"(hi.y), "=r"(hi.z), "=r"(hi.w)
+                 : "l"(p) : "memory");
+}
 
 // PLAIN: no left padding, the paper's own eviction rule, no counting of moved rows -- the instance the common case
 // runs, free of those branches.
@@ -118,13 +128,14 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
     st_global_16(dst, ld_global_16(src));
   }
   for (int j = tid; j < n1t; j += kThreads) s.id[j] = (j < c.n_old) ? c.kv_ids[base + j] : a.pos;
-  // q fragments: thread (gid, tq) holds, for every 32-element round, the 8 elements [32r + 8tq, +8) of head gid
+  // q fragments: thread (gid, tq) holds, for every pair of rounds (2R, 2R+1), the 16 elements [64R + 16tq, +16) of
+  // head gid -- the k-slots of an MMA may stand for any elements as long as both operands agree
   uint32_t qf[QR][4];
   {
     const T* qp = reinterpret_cast<const T*>(a.q) + ((size_t)smp * c.Hq + kh * G + gid) * D;
 #pragma unroll
     for (int r = 0; r < QR; ++r) {
-      const uint4 w = ldg16_or_zero(qp + 32 * r + 8 * tq, gid < G);
+      const uint4 w = ldg16_or_zero(qp + 64 * (r >> 1) + 16 * tq + 8 * (r & 1), gid < G);
       qf[r][0] = w.x; qf[r][1] = w.y; qf[r][2] = w.z; qf[r][3] = w.w;
     }
   }
@@ -136,9 +147,9 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
   auto load_k = [&](int it, uint4 (&xx)[QR], uint4 (&yy)[QR]) {
     const int j0 = it * kRowsPerIter + warp * 16 + gid, j1 = j0 + 8;
 #pragma unroll
-    for (int r = 0; r < QR; ++r) {
-      xx[r] = ldg16_or_zero(kslab + (size_t)j0 * D + 32 * r + 8 * tq, j0 < n1);
-      yy[r] = ldg16_or_zero(kslab + (size_t)j1 * D + 32 * r + 8 * tq, j1 < n1);
+    for (int R = 0; R < QR / 2; ++R) {   // elements [64R + 16tq, +16) of both rows, 32 bytes per load
+      ldg32_or_zero(kslab + (size_t)j0 * D + 64 * R + 16 * tq, j0 < n1, xx[2 * R], xx[2 * R + 1]);
+      ldg32_or_zero(kslab + (size_t)j1 * D + 64 * R + 16 * tq, j1 < n1, yy[2 * R], yy[2 * R + 1]);
     }
   };
   // rows of V for iteration `it`: thread (gid, tq) loads, from the 4 rows tb + 4tq + {0..3}, elements [64r + 8gid, +8)
