@@ -152,6 +152,15 @@ def test_extreme_decoding_arm_on_gpu(dtype, d, kv_bar):
     assert st["calls"] == len(calls)
 
 
+@pytest.mark.parametrize("g", [1, 4])
+def test_decode_with_more_caches_than_two_ctas_per_sm(g):
+    # 320 caches: the decode kernel takes its 128-thread shape (four CTAs per SM); fewer caches take the 256-thread one
+    wl = tiny("many_units", b=40, Hq=8 * g, Hkv=8, s=160, B=64, K=72, steps=10, dtype="bf16", d=128)
+    units = [(0, 0), (13, 5), (39, 7), (27, 2)]
+    st = run_lockstep(wl, units, check_rows_every=2)
+    assert st["evictions"] >= len(units) * 10
+
+
 # ------------------------------------------------------------------ the rules of Sec. 2 on the same kernels
 @pytest.mark.parametrize("rule", ["sum_recent", "current_query"])
 @pytest.mark.parametrize("dtype,d,Hq,Hkv", [("bf16", 128, 8, 2), ("f32", 64, 4, 4)])
