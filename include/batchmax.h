@@ -120,7 +120,9 @@ bm_status_t bm_cache_destroy(bm_cache_t* cache); /* frees the host handle only *
  * The block's K/V are read from the caller's buffers (they are not staged in the cache first), so the
  * call needs min(n + I, evict_to if evicting) <= cap, not n + I <= cap.
  * Errors: BM_ERR_INVALID (range, I < 1, I > block_max, null, misaligned), BM_ERR_STATE (pos0 !=
- * curr_id + 1, or the samples of the range hold different n), BM_ERR_CAPACITY. */
+ * curr_id + 1, or the samples of the range hold different n), BM_ERR_CAPACITY (the row limit above, more
+ * than 12288 candidates per cache, or more than 65535 caches -- nsamples * Hkv -- in one call: split the
+ * batch into sample ranges). */
 bm_status_t bm_prefill_block(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples,
                              const void* q, const void* k, const void* v, int32_t I, int32_t pos0,
                              void* out, int32_t evict_to, void* cuda_stream);

@@ -267,6 +267,7 @@ bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int3
   if (q == nullptr || k == nullptr || v == nullptr || out == nullptr) return BM_ERR_INVALID;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return BM_ERR_INVALID;
   if (I < 1 || I > c->cfg.block_max) return BM_ERR_INVALID;
+  if ((long long)nsamples * c->cfg.n_kv_heads > 65535) return BM_ERR_CAPACITY;   // caches of a call index grid.y
   if (pos0 != curr + 1) return BM_ERR_STATE;
   const int n_c = n_old + I;
   const int target = (evict_to >= 0 && n_c > evict_to) ? evict_to : n_c;
@@ -396,6 +397,7 @@ static bm_status_t host_pass(bm_cache_t* c, int layer, int sample0, int nsamples
   if (q == nullptr || k == nullptr || v == nullptr || out == nullptr || staging == nullptr) return BM_ERR_INVALID;
   if (reinterpret_cast<uintptr_t>(staging) & 255u) return BM_ERR_INVALID;
   if (I < 1 || I > c->cfg.block_max) return BM_ERR_INVALID;
+  if ((long long)nsamples * c->cfg.n_kv_heads > 65535) return BM_ERR_CAPACITY;   // caches of a call index grid.y
   size_t oq, ok, ov, oo, total, qb, kb;
   staging_layout(&c->cfg, nsamples, I, &oq, &ok, &ov, &oo, &total, &qb, &kb);
   if (staging_bytes < total) return BM_ERR_OOM;

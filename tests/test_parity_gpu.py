@@ -281,6 +281,16 @@ def test_error_codes_and_state_tracking():
     assert cache.length(sample=0) == cache.length(sample=1) == (wl.K, 95)
     assert cache.status() == 0
     cache.close()
+    # more caches in one prefill call than the launch grid can index: refused before anything is enqueued
+    big = bm.BatchMaxCache(bm.Config(batch=8200, n_q_heads=8, n_kv_heads=8, head_dim=64, kv_max=4, block_max=2, dtype="bf16"))
+    qb = torch.zeros(8200, 1, 8, 64, device="cuda", dtype=torch.bfloat16)
+    with pytest.raises(bm.BMError) as e:
+        big.prefill_block(qb, qb, qb, 0)
+    assert e.value.code == 3
+    big.prefill_block(qb[:4096], qb[:4096], qb[:4096], 0, sample0=0)
+    big.prefill_block(qb[4096:], qb[4096:], qb[4096:], 0, sample0=4096)
+    assert big.length(sample=8199) == (1, 0) and big.status() == 0
+    big.close()
 
 
 def test_bounded_wait_times_out_and_context_survives():
