@@ -124,8 +124,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
   // running (so that the launch latency of back-to-back decode steps is hidden); nothing that the predecessor may
   // have written -- the cache, and the inputs too -- is touched before this point.  The grid that follows may be
   // started right away: it waits at the same point for this one to complete.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  pdl_wait();
+  pdl_release();
 
   // the step's pair -> row n_old of the cache; ids -> smem
   if (tid < 2 * (D / 8)) {
@@ -450,17 +450,7 @@ cudaError_t launch_nt_p(const CacheView& c, const DecodeArgs& a, cudaStream_t st
   static SmemConfigured configured;
   if (cudaError_t err = configured.ensure(decode_mma_kernel<D, G, NT, PLAIN>, smem); err != cudaSuccess) return err;
   ProfileScope prof(kDecode, st);
-  cudaLaunchConfig_t lc = {};
-  lc.gridDim = dim3(c.nsamples * c.Hkv);
-  lc.blockDim = dim3(NT);
-  lc.dynamicSmemBytes = smem;
-  lc.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  lc.attrs = attr;
-  lc.numAttrs = 1;
-  const cudaError_t err = cudaLaunchKernelEx(&lc, decode_mma_kernel<D, G, NT, PLAIN>, c, a);
+  const cudaError_t err = launch_dependent(decode_mma_kernel<D, G, NT, PLAIN>, dim3(c.nsamples * c.Hkv), dim3(NT), smem, st, c, a);
   count_launch();
   return err != cudaSuccess ? err : cudaGetLastError();
 }
