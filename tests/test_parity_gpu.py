@@ -373,6 +373,50 @@ def test_bitwise_reproducible_and_variants_agree(dtype, d):
     assert_same_run(base, run_free(wl, micro=1))        # sample ranges: micro-batched calls
 
 
+def test_cuda_graph_replay_matches_eager_launches():
+    # the benchmark replays one CUDA graph per step; a captured schedule must leave the same bits as eager launches
+    wl = tiny("graph", b=4, dtype="bf16", d=128, Hq=8, Hkv=2, s=256, B=64, K=64, steps=6)
+    eager_outs, eager_state = run_free(wl)
+    cfg = make_config(wl)
+    inp = Inputs(wl, "cuda")
+    calls = schedule(wl)
+    ins, outs = [], []
+    for kind, pos0, I, ev in calls:
+        q, k, v = inp.block(0, pos0, I)
+        if kind == "decode":
+            q, k, v = q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()
+        ins.append((q, k, v))
+        outs.append(torch.empty_like(q))
+    arena = torch.empty(bm.arena_bytes(cfg), dtype=torch.uint8, device="cuda")
+    workspace = torch.empty(max(bm.workspace_bytes(cfg), 256), dtype=torch.uint8, device="cuda")
+
+    def step():
+        cache = bm.BatchMaxCache(cfg, arena=arena, workspace=workspace)
+        for (kind, pos0, I, ev), (q, k, v), o in zip(calls, ins, outs):
+            if kind == "prefill":
+                cache.prefill_block(q, k, v, pos0, out=o, evict_to=ev)
+            else:
+                cache.decode_step(q, k, v, out=o, evict_to=ev)
+        return cache
+
+    step().close()                       # first use of every kernel outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        captured = step()
+    for _ in range(2):                   # a replay starts from the re-created (zeroed) cache
+        graph.replay()
+    torch.cuda.synchronize()
+    for o, ref in zip(outs, eager_outs):
+        assert torch.equal(o.cpu(), ref)
+    state = [captured.export(0, s_, h, rows=True) for s_ in range(wl.b) for h in range(wl.Hkv)]
+    for sa, sb in zip(state, eager_state):
+        for x, y in zip(sa, sb):
+            assert torch.equal(x, y)
+    assert captured.status() == 0
+    captured.close()
+
+
 def test_export_import_roundtrip_resumes_identically():
     wl = tiny("ckpt", dtype="bf16", d=128, Hq=8, Hkv=2, s=192, B=64, K=48, steps=0)
     cfg = make_config(wl)
