@@ -373,9 +373,12 @@ def test_bitwise_reproducible_and_variants_agree(dtype, d):
     assert_same_run(base, run_free(wl, micro=1))        # sample ranges: micro-batched calls
 
 
-def test_cuda_graph_replay_matches_eager_launches():
+@pytest.mark.parametrize("which", ["tiny", "cfg2"])
+def test_cuda_graph_replay_matches_eager_launches(which):
     # the benchmark replays one CUDA graph per step; a captured schedule must leave the same bits as eager launches
-    wl = tiny("graph", b=4, dtype="bf16", d=128, Hq=8, Hkv=2, s=256, B=64, K=64, steps=6)
+    # (which the lock-step tests hold against the oracle) -- also at the benchmark's own full size
+    wl = tiny("graph", b=4, dtype="bf16", d=128, Hq=8, Hkv=2, s=256, B=64, K=64, steps=6) if which == "tiny" \
+        else WORKLOADS["cfg2"]
     eager_outs, eager_state = run_free(wl)
     cfg = make_config(wl)
     inp = Inputs(wl, "cuda")
