@@ -226,7 +226,7 @@ def main():
         dist.barrier()
     import paper_2412_05693_b200 as bm
     from paper_2412_05693_b200.workloads import Inputs, schedule
-    from tests.lockstep import make_config
+    from paper_2412_05693_b200.workloads import config_for as make_config
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     calls = schedule(wl)

@@ -16,7 +16,7 @@ import torch
 
 from oracle import UnitCache
 from paper_2412_05693_b200 import BatchMaxCache, Config
-from paper_2412_05693_b200.workloads import Inputs, Workload, schedule
+from paper_2412_05693_b200.workloads import Inputs, Workload, config_for, schedule
 
 BAND = 1e-4   # relative band around the cut inside which kept sets may differ
 OUT_TOL = {"bf16": 2e-2, "f32": 1e-4}
@@ -24,9 +24,7 @@ OUT_TOL = {"bf16": 2e-2, "f32": 1e-4}
 
 def make_config(wl: Workload, device: int = 0, growth: int | None = None, batch: int | None = None,
                 max_call_samples: int = 0, rule: str = "average") -> Config:
-    return Config(batch=wl.b if batch is None else batch, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.d,
-                  kv_max=wl.K, block_max=wl.B, growth=max(1, wl.p_dec) if growth is None else growth,
-                  dtype=wl.dtype, n_layers=wl.L, device=device, max_call_samples=max_call_samples, rule=rule)
+    return config_for(wl, device, growth, batch, max_call_samples, rule)
 
 
 def _np(t):

@@ -116,3 +116,17 @@ def test_product_package_does_not_import_the_oracle():
                 src = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in src.lower() or f == "workloads.py", f
     assert "import oracle" not in open(os.path.join(pkg, "workloads.py")).read()
+
+
+def test_benchmark_reaches_the_oracle_only_in_its_cpu_legs():
+    # importing the benchmark (and everything its GPU arm imports at module level) must not load the oracle;
+    # the oracle is imported inside the CPU-baseline / reference-arm function only
+    import subprocess
+    import sys
+    code = ("import sys; sys.path.insert(0, %r); import bench, paper_2412_05693_b200, "
+            "paper_2412_05693_b200.workloads, paper_2412_05693_b200.experiments; "
+            "assert not any(m == 'oracle' or m.startswith('oracle.') for m in sys.modules), 'oracle imported'; "
+            "assert not any(m.startswith('tests') for m in sys.modules), 'tests imported'") % ROOT
+    subprocess.run([sys.executable, "-c", code], check=True, cwd=ROOT)
+    src = open(os.path.join(ROOT, "bench.py")).read()
+    assert src.count("from oracle import") == 1 and "tests.lockstep" not in src
