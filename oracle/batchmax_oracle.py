@@ -162,6 +162,7 @@ class UnitCache:
             window = int(target) // 2
             if window > 0:
                 score[len(self) - window:] = np.inf
+            score[self.kv_ids < self.left_pad] = 0.0   # padding is never "recent": it ranks last whatever its position
         return score
 
     def evict(self, target: int, curr_id: int | None = None, kept_ids=None):

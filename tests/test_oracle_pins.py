@@ -629,3 +629,16 @@ def test_sum_recent_keeps_its_window_and_current_query_forgets():
     np.testing.assert_allclose(u2.sum_weights, w[19, 0], rtol=1e-14)   # the last query's row and nothing else
     u2.decode_step(q[20], k[20], v[20])
     assert u2.sum_weights.sum() == pytest.approx(1.0)             # previous sums are gone
+
+
+def test_padding_ranks_last_even_inside_the_recent_window():
+    # a block that is all padding: the window of the most recent candidates holds padding only, which still
+    # leaves from the top, so the lowest padding positions are what stays
+    g, d = 1, 4
+    q, k, v = rand_qkv(71, 40, g, d)
+    u = UnitCache(d, g, left_pad=30, rule="sum_recent")
+    u.process_block(q[:20], k[:20], v[:20], 0, evict_to=8)
+    assert u.kv_ids.tolist() == list(range(8))
+    u.process_block(q[20:40], k[20:40], v[20:40], 20, evict_to=8)     # 10 more padding positions, then 10 real ones
+    assert u.kv_ids.tolist()[-4:] == [36, 37, 38, 39]                  # the window of recent real pairs
+    assert all(i >= 30 for i in u.kv_ids.tolist())                     # every real pair outranks padding

@@ -170,6 +170,13 @@ def test_alternative_eviction_rules_lockstep(rule, dtype, d, Hq, Hkv):
     assert st["evictions"] >= 2 * Hkv * (3 + 12)
 
 
+def test_alternative_rule_with_left_padding():
+    # first blocks entirely padding: the recent window holds padding, which still ranks last
+    wl = tiny("rules_pad", b=3, s=320, B=64, K=40, steps=6, dtype="bf16", d=128, Hq=8, Hkv=2)
+    run_lockstep(wl, all_units(wl), rule="sum_recent", pads=[0, 100, 300], check_rows_every=2)
+    run_lockstep(wl, all_units(wl), rule="current_query", pads=[5, 64, 250], check_rows_every=2)
+
+
 def test_alternative_rule_with_growth_falls_back_to_the_general_select():
     # decode evicts 8 pairs at a time: the fused arg-min does not apply, the select kernel ranks by the rule
     wl = tiny("rules_g", s=256, B=64, K=64, steps=20, p_dec=8, dtype="bf16", d=128, Hq=8, Hkv=2)
