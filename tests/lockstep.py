@@ -34,6 +34,11 @@ def _np(t):
 def check_kept(unit: UnitCache, gpu_ids: np.ndarray, target: int, stats: dict, where: str):
     """Band check of the GPU's kept set against the oracle's ranking; the oracle then evicts (adopting the
     GPU's set when it differs inside the band)."""
+    if target == 0:                               # everything leaves: nothing to rank
+        assert len(gpu_ids) == 0, f"{where}: {len(gpu_ids)} pairs kept, target 0"
+        unit.evict(0)
+        stats["evictions"] += 1
+        return
     ave = unit.ranking_scores(target)             # ave_weights under the paper's rule
     cand = unit.kv_ids
     is_pad = cand < unit.left_pad                 # padding pairs of a left-padded sample rank after every real pair
@@ -117,7 +122,8 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
             n_gpu, cur = cache.length(layer, smp)
             assert n_gpu == len(unit) and cur == unit.last_pos, f"{where}: host mirror n/curr_id wrong"
             sw = sw.numpy().astype(np.float64)
-            rel = float(np.max(np.abs(sw - unit.sum_weights) / np.maximum(np.abs(unit.sum_weights), 1e-3)))
+            rel = float(np.max(np.abs(sw - unit.sum_weights) / np.maximum(np.abs(unit.sum_weights), 1e-3))) \
+                if len(unit) else 0.0              # (an eviction call on a still-empty cache is legal)
             stats["max_sum_rel"] = max(stats["max_sum_rel"], rel)
             assert rel <= sum_rtol, f"{where}: sum_weights relative error {rel:.3e} > {sum_rtol}"
             if want_rows:

@@ -98,6 +98,42 @@ def test_random_shapes(wl):
     assert st["calls"] == len(schedule(wl))
 
 
+def random_cadence(wl, rng):
+    """The workload's schedule with evictions switched off at random, explicit bm_evict / bm_keep_most_recent calls
+    (targets from 0 up) thrown in, and an eviction forced wherever the cache would overflow."""
+    growth = wl.B + 5
+    calls, n = [], 0
+    for kind, pos0, I, ev in schedule(wl):
+        if n + I > wl.K + growth - 1 or rng.random() < 0.3:
+            tgt = int(rng.integers(0, wl.K + 1))
+            calls.append(("recent" if rng.random() < 0.3 else "evict", 0, 0, tgt))
+            n = min(n, tgt)
+        use_ev = ev if rng.random() < 0.5 else -1
+        if use_ev < 0 and n + I > wl.K + growth:
+            use_ev = wl.K
+        calls.append((kind, pos0, I, use_ev))
+        n = n + I if use_ev < 0 else min(n + I, use_ev)
+    return calls, growth
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_cadences_rules_and_padding(seed):
+    # seeded samples of the randomised sweep this suite was hardened with: any cadence of the four calls, any rule,
+    # left padding, evictions down to an empty cache
+    rng = np.random.default_rng(4200 + seed)
+    g, hkv, d = int(rng.choice([1, 2, 4, 8])), int(rng.integers(1, 4)), int(rng.choice([64, 128]))
+    wl = Workload(f"cad{seed}", b=int(rng.integers(1, 4)), Hq=g * hkv, Hkv=hkv, d=d, dtype=str(rng.choice(["bf16", "f32"])),
+                  s=int(rng.integers(50, 900)), B=int(rng.integers(1, 300)), K=int(rng.integers(1, 400)),
+                  steps=int(rng.integers(0, 16)), seed=4200 + seed, heavy_count=3, p_dec=int(rng.choice([1, 3])))
+    rule = str(rng.choice(["average", "sum_recent", "current_query"]))
+    if seed % 2 == 0:
+        calls, growth = random_cadence(wl, rng)
+        run_lockstep(wl, all_units(wl)[:3], calls=calls, growth=growth, rule=rule, check_rows_every=3)
+    else:
+        pads = [int(rng.integers(0, wl.s + 1)) for _ in range(wl.b)]
+        run_lockstep(wl, all_units(wl)[:3], pads=pads, rule=rule, check_rows_every=3)
+
+
 # ------------------------------------------------------------------ shapes, tails and degenerate cases
 @pytest.mark.parametrize("wl", [
     tiny("ragged_f32"),                                               # I = 48, tail of 8, g = 2
