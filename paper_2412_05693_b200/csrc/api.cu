@@ -5,6 +5,7 @@
 #include <cstring>
 #include <new>
 #include <utility>
+#include <algorithm>
 #include <vector>
 
 #include "../../include/batchmax.h"
@@ -100,6 +101,11 @@ struct bm_cache {
   float* ws_new_sum;
   int32_t* left_pad = nullptr;   // [batch] device copy of the samples' padding counts (in the workspace)
   bool has_pad = false;          // some sample is left-padded
+  // Padding leaves first at every eviction (under every rule), so how many padding pairs a sample's caches still
+  // hold is a function of the calls made: the host tracks it and takes the kernels' padding-free instances again as
+  // soon as a call's samples hold none and its block lies behind their padding.
+  std::vector<int32_t> pad_host;  // [batch]
+  std::vector<int32_t> npad;      // [L * b] padding pairs cached (kNpadUnknown after an import / set_len)
   bool count_moves = false;      // compactions add the rows they move to the counters in the status block
   std::vector<int32_t> n, curr_id;  // [L * b] host mirror
   // host-fed calls run as a three-stage pipeline on streams owned by the handle -- input copies, the pass,
@@ -138,7 +144,31 @@ bm_status_t check_range(const bm_cache* c, int layer, int sample0, int nsamples,
   return BM_OK;
 }
 
-CacheView make_view(const bm_cache* c, int layer, int sample0, int nsamples, int n_old) {
+constexpr int32_t kNpadUnknown = 1 << 30;
+
+// Does a call on this range, whose new pairs occupy positions [pos0, pos0 + I), meet any padding?
+bool pad_active(const bm_cache* c, int layer, int sample0, int nsamples, int pos0, int I) {
+  if (!c->has_pad) return false;
+  const size_t o = (size_t)layer * c->cfg.batch + sample0;
+  for (int s = 0; s < nsamples; ++s)
+    if (c->npad[o + s] > 0 || (I > 0 && pos0 < c->pad_host[sample0 + s])) return true;
+  return false;
+}
+
+// After a call that appended the positions [pos0, pos0 + I) and then removed `removed` pairs.
+void pad_update(bm_cache* c, int layer, int sample0, int nsamples, int pos0, int I, int removed) {
+  if (!c->has_pad) return;
+  const size_t o = (size_t)layer * c->cfg.batch + sample0;
+  for (int s = 0; s < nsamples; ++s) {
+    int32_t& np = c->npad[o + s];
+    if (np >= kNpadUnknown) continue;
+    const int pad = c->pad_host[sample0 + s];
+    const int added = I > 0 ? std::max(0, std::min(I, pad - pos0)) : 0;
+    np = std::max(0, np + added - removed);
+  }
+}
+
+CacheView make_view(const bm_cache* c, int layer, int sample0, int nsamples, int n_old, bool with_pad = true) {
   CacheView v;
   const size_t unit0 = ((size_t)layer * c->cfg.batch + sample0) * c->cfg.n_kv_heads;
   const size_t row0 = unit0 * c->cap;
@@ -153,7 +183,7 @@ CacheView make_view(const bm_cache* c, int layer, int sample0, int nsamples, int
   v.g = c->g;
   v.nsamples = nsamples;
   v.status = c->status;
-  v.left_pad = c->has_pad ? c->left_pad + sample0 : nullptr;
+  v.left_pad = (c->has_pad && with_pad) ? c->left_pad + sample0 : nullptr;
   v.rule = c->cfg.rule;
   v.moved = c->count_moves ? reinterpret_cast<unsigned long long*>(c->status + 16) : nullptr;
   return v;
@@ -276,7 +306,7 @@ bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int3
   if ((s = set_device(c)) != BM_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
-  CacheView view = make_view(c, layer, sample0, nsamples, n_old);
+  CacheView view = make_view(c, layer, sample0, nsamples, n_old, pad_active(c, layer, sample0, nsamples, pos0, I));
   BlockArgs a;
   a.q = q; a.k = k; a.v = v; a.out = out;
   a.lse = c->ws_lse; a.new_sum = c->ws_new_sum;
@@ -304,6 +334,7 @@ bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int3
     n_new = target;
   }
   set_mirror(c, layer, sample0, nsamples, n_new, pos0 + I - 1);
+  pad_update(c, layer, sample0, nsamples, pos0, I, n_c - n_new);
   return BM_OK;
 }
 
@@ -324,8 +355,8 @@ bm_status_t bm_decode_step(bm_cache_t* c, int32_t layer, int32_t sample0, int32_
   if (n1 > kMaxCandidates || smem > kMaxSmem) return BM_ERR_CAPACITY;
   if ((s = set_device(c)) != BM_OK) return s;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  CacheView view = make_view(c, layer, sample0, nsamples, n_old);
   const int pos = curr + 1;
+  CacheView view = make_view(c, layer, sample0, nsamples, n_old, pad_active(c, layer, sample0, nsamples, pos, 1));
   // target 0: nothing survives -- run the attention and the update, then empty the caches on the host mirror
   const int kernel_target = target == 0 ? -1 : target;
   const cudaError_t err = mma ? launch_decode_mma(c->cfg.head_dim, view, q, k, v, out, pos, c->scale, kernel_target, st)
@@ -334,6 +365,7 @@ bm_status_t bm_decode_step(bm_cache_t* c, int32_t layer, int32_t sample0, int32_
   if (err != cudaSuccess) return BM_ERR_CUDA;
   const int n_new = target >= 0 ? target : n1;
   set_mirror(c, layer, sample0, nsamples, n_new, pos);
+  pad_update(c, layer, sample0, nsamples, pos, 1, n1 - n_new);
   return BM_OK;
 }
 
@@ -345,15 +377,22 @@ static bm_status_t evict_cached(bm_cache_t* c, int32_t layer, int32_t sample0, i
   ++c->dev_calls;  // a later host-fed call orders its pipeline after this one
   if (target < 0) return BM_ERR_INVALID;
   if (n_old <= target) return BM_OK;
-  if (target == 0) { set_mirror(c, layer, sample0, nsamples, 0, curr); return BM_OK; }
+  if (target == 0) {
+    set_mirror(c, layer, sample0, nsamples, 0, curr);
+    pad_update(c, layer, sample0, nsamples, 0, 0, n_old);
+    if (c->has_pad)                                   // an empty cache holds no padding, whatever was unknown before
+      for (int s2 = 0; s2 < nsamples; ++s2) c->npad[(size_t)layer * c->cfg.batch + sample0 + s2] = 0;
+    return BM_OK;
+  }
   if (n_old > kMaxCandidates) return BM_ERR_CAPACITY;
   if ((s = set_device(c)) != BM_OK) return s;
-  CacheView view = make_view(c, layer, sample0, nsamples, n_old);
+  CacheView view = make_view(c, layer, sample0, nsamples, n_old, pad_active(c, layer, sample0, nsamples, 0, 0));
   EvictArgs e;
   e.blk_k = nullptr; e.blk_v = nullptr; e.new_sum = nullptr;
   e.I = 0; e.pos0 = 0; e.curr_id = curr; e.target = target; e.recent = recent ? 1 : 0;
   if ((s = run_evict(c, view, e, static_cast<cudaStream_t>(cuda_stream))) != BM_OK) return s;
   set_mirror(c, layer, sample0, nsamples, target, curr);
+  pad_update(c, layer, sample0, nsamples, 0, 0, n_old - target);   // both rules remove padding before anything else
   return BM_OK;
 }
 
@@ -509,6 +548,8 @@ bm_status_t bm_cache_set_left_pad(bm_cache_t* c, const int32_t* pads, void* cuda
     }
   c->has_pad = any;
   if (!any) return BM_OK;
+  c->pad_host.assign(pads, pads + c->cfg.batch);
+  c->npad.assign((size_t)c->cfg.n_layers * c->cfg.batch, 0);
   bm_status_t st = set_device(c);
   if (st != BM_OK) return st;
   ++c->dev_calls;
@@ -548,6 +589,7 @@ bm_status_t bm_cache_set_len(bm_cache_t* c, int32_t layer, int32_t sample, int32
   const size_t o = (size_t)layer * c->cfg.batch + sample;
   c->n[o] = n;
   c->curr_id[o] = curr_id;
+  if (c->has_pad) c->npad[o] = n > 0 ? kNpadUnknown : 0;   // contents come from outside: assume padding may be there
   return BM_OK;
 }
 
