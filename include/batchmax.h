@@ -181,8 +181,8 @@ bm_status_t bm_prefill_block_static(bm_cache_t* cache, int32_t layer, int32_t sa
  * and later work on cuda_stream sees the updated cache).  The pipeline is ordered after cuda_stream's
  * position only where it has to be: at the first host-fed call and after any device-fed call on this
  * handle.  The input copies start at call time, so q/k/v must hold their final contents when the call
- * is made and until cuda_stream has passed the call.  Passing two staging buffers alternately keeps two
- * calls in flight; a staging buffer is reused only after the earlier call that used it has finished
+ * is made and until cuda_stream has passed the call.  Passing up to four staging buffers in turn keeps as
+ * many calls in flight; a staging buffer is reused only after the earlier call that used it has finished
  * (tracked by the handle).  While cuda_stream is being captured into a CUDA graph everything stays on
  * cuda_stream. */
 bm_status_t bm_staging_bytes(const bm_config_t* cfg /*HOST*/, int32_t nsamples, int32_t I, size_t* bytes);

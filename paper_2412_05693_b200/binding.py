@@ -286,13 +286,13 @@ class BatchMaxCache:
 
     # -- host-fed variants ---------------------------------------------------------------------------
     def _stage(self, ns, I):
-        """Two staging buffers used alternately, so that consecutive host-fed calls overlap their copies."""
+        """Four staging buffers used in turn, so that consecutive host-fed calls overlap their copies and passes."""
         need = staging_bytes(self.cfg, ns, I)
         if self._staging is None or self._staging[0].numel() < need:
             dev = self.torch.device("cuda", self.cfg.device)
-            self._staging = [self.torch.empty(need, dtype=self.torch.uint8, device=dev) for _ in range(2)]
+            self._staging = [self.torch.empty(need, dtype=self.torch.uint8, device=dev) for _ in range(4)]
             self._stage_turn = 0
-        self._stage_turn ^= 1
+        self._stage_turn = (self._stage_turn + 1) % 4
         return self._staging[self._stage_turn]
 
     def prefill_block_host(self, q, k, v, pos0: int, out, evict_to: int = -1, layer: int = 0, sample0: int = 0,

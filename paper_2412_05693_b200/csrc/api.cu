@@ -110,14 +110,15 @@ struct bm_cache {
   std::vector<int32_t> n, curr_id;  // [L * b] host mirror
   // host-fed calls run as a three-stage pipeline on streams owned by the handle -- input copies, the pass,
   // the output copy -- so that the three stages of consecutive calls overlap (PCIe is full duplex); the
-  // caller's stream only waits for each call's output copy.  Two staging buffers can be in flight.
+  // caller's stream only waits for each call's output copy.  Up to four staging buffers can be in flight.
   cudaStream_t in_stream = nullptr, work_stream = nullptr, out_stream = nullptr;
   cudaEvent_t entry_ev = nullptr;
   struct Slot {
     void* staging = nullptr;
     cudaEvent_t in_done = nullptr, pass_done = nullptr, call_done = nullptr;
   };
-  Slot slots[2];
+  static constexpr int kSlots = 4;
+  Slot slots[kSlots];
   int next_slot = 0;
   long dev_calls = 0, dev_calls_seen = -1;  // device-fed calls made / already ordered before the pipeline
 };
@@ -471,7 +472,7 @@ static bm_status_t host_pass(bm_cache_t* c, int layer, int sample0, int nsamples
     }
     for (auto& sl : c->slots)
       if (sl.staging == staging) slot = &sl;
-    if (slot == nullptr) { slot = &c->slots[c->next_slot]; c->next_slot ^= 1; }
+    if (slot == nullptr) { slot = &c->slots[c->next_slot]; c->next_slot = (c->next_slot + 1) % bm_cache::kSlots; }
     in = c->in_stream;
     work = c->work_stream;
     outs = c->out_stream;
