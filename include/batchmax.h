@@ -92,8 +92,8 @@ bm_status_t bm_cache_bytes_per_sample(const bm_config_t* cfg /*HOST*/, size_t* b
 bm_status_t bm_arena_bytes(const bm_config_t* cfg /*HOST*/, size_t* bytes /*HOST out*/);
 /* Largest batch whose arena fits in hbm_budget_bytes (cfg->batch is ignored); 0 if none fits. */
 bm_status_t bm_max_batch(const bm_config_t* cfg /*HOST*/, size_t hbm_budget_bytes, int32_t* b /*HOST out*/);
-/* Per-call scratch (log-sum-exp of every query row and the new pairs' column sums) for calls of up
- * to max_call_samples samples and block_max inputs. */
+/* Scratch of a handle: per call, the log-sum-exp of every query row and the new pairs' column sums, for calls of
+ * up to max_call_samples samples and block_max inputs; plus one padding count per sample (bm_cache_set_left_pad). */
 bm_status_t bm_workspace_bytes(const bm_config_t* cfg /*HOST*/, size_t* bytes /*HOST out*/);
 
 /* Carve `arena` (DEVICE, 256-byte aligned, >= bm_arena_bytes) into the slabs
