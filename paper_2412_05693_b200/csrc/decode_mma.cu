@@ -236,24 +236,22 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
     for (int j = tid; j < n1; j += kThreads)
 #pragma unroll
       for (int h = 0; h < G; ++h) m[h] = fmaxf(m[h], s.p[h * n1t + j]);
+    // the warp's maximum first (plain max shuffles), then every lane sums relative to it: no exponentials inside
+    // the shuffle chain
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1)
+#pragma unroll
+      for (int h = 0; h < G; ++h) m[h] = fmaxf(m[h], __shfl_xor_sync(0xffffffffu, m[h], off));
 #pragma unroll
     for (int h = 0; h < G; ++h) t[h] = 0.f;
     for (int j = tid; j < n1; j += kThreads)
 #pragma unroll
-      for (int h = 0; h < G; ++h) t[h] += ex2f(s.p[h * n1t + j] - m[h]);   // ex2(-inf) = 0 when a thread has no row
+      for (int h = 0; h < G; ++h)   // a warp whose rows are all masked carries (-inf, 0): no inf - inf
+        t[h] += ex2f(s.p[h * n1t + j] - (m[h] == -INFINITY ? 0.f : m[h]));
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1)
 #pragma unroll
-      for (int h = 0; h < G; ++h) {
-        const float mo = __shfl_xor_sync(0xffffffffu, m[h], off), to = __shfl_xor_sync(0xffffffffu, t[h], off);
-        const float mn = fmaxf(m[h], mo);
-        // a side that has seen no row carries (-inf, 0): its term must not produce inf - inf
-        const float a0 = (m[h] == -INFINITY) ? 0.f : t[h] * ex2f(m[h] - mn);
-        const float a1 = (mo == -INFINITY) ? 0.f : to * ex2f(mo - mn);
-        // both lanes of a pair must add in the same order to stay bit-identical
-        t[h] = (lane & off) ? (a1 + a0) : (a0 + a1);
-        m[h] = mn;
-      }
+      for (int h = 0; h < G; ++h) t[h] += __shfl_xor_sync(0xffffffffu, t[h], off);   // a + b == b + a: lanes agree
     if (lane == 0)
 #pragma unroll
       for (int h = 0; h < G; ++h) { s.wred[h * kWarps + warp] = m[h]; s.wred[(G + h) * kWarps + warp] = t[h]; }
