@@ -693,6 +693,16 @@ bool tc_path_available() {
   return encode_fn() != nullptr;
 }
 
+// Map over the first `rows` rows of every cache of a slab, as tiles of `box_rows` rows x 64 elements (128-byte
+// swizzle); rows past `rows` read as zeros.  False when the driver's encoder is unavailable or refuses.
+bool encode_slab_rows_map(CUtensorMap* m, const void* slab, int d, int rows, int cap, int units, int box_rows) {
+  if (encode_fn() == nullptr) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)(rows > 0 ? rows : 1), (cuuint64_t)units};
+  const cuuint64_t str[2] = {(cuuint64_t)d * 2, (cuuint64_t)cap * d * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  return encode(m, slab, 3, dims, str, box);
+}
+
 cudaError_t launch_attn_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used) {
   *used = 0;
   g_maps_q = nullptr;

@@ -10,6 +10,7 @@
 #include <cstdlib>
 
 #include "evict.cuh"
+#include "tc_common.cuh"
 
 namespace bm {
 namespace {
@@ -96,10 +97,21 @@ __device__ __forceinline__ void ldg32_or_zero(const __nv_bfloat16* p, bool ok, u
                  : "l"(p) : "memory");
 }
 
+__device__ __forceinline__ void stg32(__nv_bfloat16* p, const uint4& lo, const uint4& hi) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+               :: "l"(p), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
+}
+
 // PLAIN: no left padding, the paper's own eviction rule, no counting of moved rows -- the instance the common case
 // runs, free of those branches.
-template <int D, int G, int NT, bool PLAIN>
-__global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, DecodeArgs a) {
+// KD: 1 = every warp keeps one tile of rows in flight beyond the one it multiplies (fits the register budget of two
+// or four CTAs per SM).  KD > 1 = one CTA per SM with the whole register file, for caches of at most KD tiles per
+// warp in grids of at most one CTA per SM: all of K is loaded at once and stays in registers until the pair that
+// leaves is known, so that the rows behind it are written one row up straight from registers.  Such a grid's step
+// lasts as long as its slowest CTA, which is the one that has to move most of its cache; re-reading K for the move
+// (as the KD = 1 instances do) made that CTA 4.7 us slower than the fastest one at 128 caches of 512 pairs.
+template <int D, int G, int NT, bool PLAIN, int KD>
+__global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(CacheView c, DecodeArgs a, const __grid_constant__ CUtensorMap vmap) {
   using T = __nv_bfloat16;
   constexpr int kThreads = NT, kWarps = NT / 32;
   constexpr int kRowsPerIter = kWarps * 16;   // one 16-key tile per warp and iteration
@@ -126,6 +138,15 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
   // started right away: it waits at the same point for this one to complete.
   pdl_wait();
   pdl_release();
+  if constexpr (KD > 1) {   // barriers of the V tiles (initialised by the thread that issues the copies)
+    if (tid == 0) {
+      const uint32_t st0 = (tc::smem_u32(smem_raw) + (uint32_t)smem_layout(nullptr, D, G, n1, kWarps, nullptr) + 1023u) & ~1023u;
+      unsigned char* st = smem_raw + (st0 - tc::smem_u32(smem_raw));
+      for (int u = 0; u < KD; ++u) tc::mbar_init(reinterpret_cast<uint64_t*>(st) + u, 1);
+      *reinterpret_cast<volatile int*>(st + 64) = 0;
+      tc::mbar_fence_init();
+    }
+  }
 
   // the step's pair -> row n_old of the cache; ids -> smem
   if (tid < 2 * (D / 8)) {
@@ -151,12 +172,30 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
 
   // ---- logits (log2 domain).  Tile rows gid and gid+8; the k-slots of thread tq are its own 8 elements.
   // The loads of iteration it+1 are issued before the MMAs of iteration it (one round trip in flight).
+  // (batched mode reads the step's own pair from the caller's buffers, so that no load waits for the barrier that
+  // publishes the appended row)
+  const T* k_new = reinterpret_cast<const T*>(a.k) + ((size_t)smp * c.Hkv + kh) * D;
+  const T* v_new = reinterpret_cast<const T*>(a.v) + ((size_t)smp * c.Hkv + kh) * D;
+  auto k_row = [&](int j) { return (KD > 1 && j == c.n_old) ? k_new : kslab + (size_t)j * D; };
+  auto v_row = [&](int j) { return (KD > 1 && j == c.n_old) ? v_new : vslab + (size_t)j * D; };
   auto load_k = [&](int it, uint4 (&xx)[QR], uint4 (&yy)[QR]) {
     const int j0 = it * kRowsPerIter + warp * 16 + gid, j1 = j0 + 8;
 #pragma unroll
     for (int R = 0; R < QR / 2; ++R) {   // elements [64R + 16tq, +16) of both rows, 32 bytes per load
-      ldg32_or_zero(kslab + (size_t)j0 * D + 64 * R + 16 * tq, j0 < n1, xx[2 * R], xx[2 * R + 1]);
-      ldg32_or_zero(kslab + (size_t)j1 * D + 64 * R + 16 * tq, j1 < n1, yy[2 * R], yy[2 * R + 1]);
+      ldg32_or_zero(k_row(j0) + 64 * R + 16 * tq, j0 < n1, xx[2 * R], xx[2 * R + 1]);
+      ldg32_or_zero(k_row(j1) + 64 * R + 16 * tq, j1 < n1, yy[2 * R], yy[2 * R + 1]);
+    }
+  };
+  auto store_logits = [&](int it, const float (&cacc)[4]) {
+    // cacc[0], cacc[1]: key j0, heads 2tq, 2tq+1 ; cacc[2], cacc[3]: key j1
+    const int j0 = it * kRowsPerIter + warp * 16 + gid, j1 = j0 + 8;
+    if (2 * tq < G) {
+      if (j0 < n1) s.p[(2 * tq) * n1t + j0] = cacc[0] * sc2;
+      if (j1 < n1) s.p[(2 * tq) * n1t + j1] = cacc[2] * sc2;
+    }
+    if (2 * tq + 1 < G) {
+      if (j0 < n1) s.p[(2 * tq + 1) * n1t + j0] = cacc[1] * sc2;
+      if (j1 < n1) s.p[(2 * tq + 1) * n1t + j1] = cacc[3] * sc2;
     }
   };
   // rows of V for iteration `it`: thread (gid, tq) loads, from the 4 rows tb + 4tq + {0..3}, elements [64r + 8gid, +8)
@@ -166,9 +205,25 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
     for (int r = 0; r < VR; ++r)
 #pragma unroll
       for (int sx = 0; sx < 4; ++sx)
-        zz[r][sx] = ldg16_or_zero(vslab + (size_t)(jr + sx) * D + 64 * r + 8 * gid, jr + sx < n1);
+        zz[r][sx] = ldg16_or_zero(v_row(jr + sx) + 64 * r + 8 * gid, jr + sx < n1);
   };
-  {
+  uint4 xk[KD > 1 ? KD : 1][QR], yk[KD > 1 ? KD : 1][QR];   // KD > 1: the whole cache's K rows (n_iter <= KD)
+  if constexpr (KD > 1) {
+#pragma unroll
+    for (int u = 0; u < KD; ++u) load_k(u, xk[u], yk[u]);   // tiles beyond the last hold no row: no load issued
+#pragma unroll
+    for (int u = 0; u < KD; ++u) {
+      if (u < n_iter) {
+        float cacc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int r = 0; r < QR; ++r) {
+          mma16816(cacc, xk[u][r].x, yk[u][r].x, xk[u][r].y, yk[u][r].y, qf[r][0], qf[r][1]);
+          mma16816(cacc, xk[u][r].z, yk[u][r].z, xk[u][r].w, yk[u][r].w, qf[r][2], qf[r][3]);
+        }
+        store_logits(u, cacc);
+      }
+    }
+  } else {
     uint4 x[QR], y[QR];
     // the first tile of K does not contain the row appended above unless the cache is still tiny, so its loads
     // are issued before the barrier that publishes that row
@@ -177,7 +232,6 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
     __syncthreads();
     if (!early) load_k(0, x, y);
     for (int it = 0; it < n_iter; ++it) {
-      const int j0 = it * kRowsPerIter + warp * 16 + gid, j1 = j0 + 8;
       uint4 xn[QR], yn[QR];
       if (it + 1 < n_iter) load_k(it + 1, xn, yn);
       float cacc[4] = {0.f, 0.f, 0.f, 0.f};
@@ -186,15 +240,7 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
         mma16816(cacc, x[r].x, y[r].x, x[r].y, y[r].y, qf[r][0], qf[r][1]);
         mma16816(cacc, x[r].z, y[r].z, x[r].w, y[r].w, qf[r][2], qf[r][3]);
       }
-      // cacc[0], cacc[1]: key j0, heads 2tq, 2tq+1 ; cacc[2], cacc[3]: key j1
-      if (2 * tq < G) {
-        if (j0 < n1) s.p[(2 * tq) * n1t + j0] = cacc[0] * sc2;
-        if (j1 < n1) s.p[(2 * tq) * n1t + j1] = cacc[2] * sc2;
-      }
-      if (2 * tq + 1 < G) {
-        if (j0 < n1) s.p[(2 * tq + 1) * n1t + j0] = cacc[1] * sc2;
-        if (j1 < n1) s.p[(2 * tq + 1) * n1t + j1] = cacc[3] * sc2;
-      }
+      store_logits(it, cacc);
       if (it + 1 < n_iter) {
 #pragma unroll
         for (int r = 0; r < QR; ++r) { x[r] = xn[r]; y[r] = yn[r]; }
@@ -203,7 +249,28 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
   }
   // first V tile and the old sum_weights start loading now; they are needed only after the softmax
   uint4 z[VR][4];
-  load_v(0, z);
+  // KD > 1: all of V starts on its way into shared memory now, as TMA tiles of 128 rows x 64 elements (128-byte
+  // swizzle; rows past n_old arrive as zeros), one mbarrier per 128 rows.  The copies stream while the softmax
+  // phases run and pass by the register file, whose write-back path those phases need (the same rows prefetched
+  // into registers made the phases longer by the time the loads took; per-thread cp.async stalled at issue).
+  const uint32_t stage0 = (tc::smem_u32(smem_raw) + (uint32_t)smem_layout(nullptr, D, G, n1, kWarps, nullptr) + 1023u) & ~1023u;
+  unsigned char* stage = smem_raw + (stage0 - tc::smem_u32(smem_raw));   // [0, 1024): barriers; then the tiles
+  uint64_t* vbar = reinterpret_cast<uint64_t*>(stage);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(stage + 64);
+  constexpr int kBoxBytes = 128 * 128;   // 128 rows x 64 bf16
+  if constexpr (KD > 1) {
+    if (tid == 0) {
+#pragma unroll
+      for (int u = 0; u < KD; ++u)
+        if (u < n_iter) {
+          tc::mbar_expect_tx(&vbar[u], 2 * kBoxBytes);
+          tc::tma_load_3d(stage + 1024 + (2 * u) * kBoxBytes, &vmap, 0, u * 128, unit, &vbar[u]);
+          tc::tma_load_3d(stage + 1024 + (2 * u + 1) * kBoxBytes, &vmap, 64, u * 128, unit, &vbar[u]);
+        }
+    }
+  } else {
+    load_v(0, z);
+  }
   constexpr int kSwPrefetch = 4;
   float sw_old[kSwPrefetch];
 #pragma unroll
@@ -347,11 +414,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
     for (int m = 0; m < 4; ++m)
 #pragma unroll
       for (int e = 0; e < 4; ++e) oacc[r][m][e] = 0.f;
-  for (int it = 0; it < n_iter; ++it) {
+  // one tile of 16 rows per warp: its MMAs, then -- once the hole lies in or before the tile -- its rows' move up
+  auto pv_tile = [&](int it, const uint4 (&zt)[VR][4]) {
     const int tb = it * kRowsPerIter + warp * 16;
     const int jr = tb + 4 * tq;   // first of this thread's 4 rows
-    uint4 zn[VR][4];
-    if (it + 1 < n_iter) load_v(it + 1, zn);   // next iteration's rows load while this one is multiplied
     // p^T fragment: (head gid; keys jr, jr+1) and (head gid; keys jr+2, jr+3)
     uint32_t pb0 = 0u, pb1 = 0u;
     if (gid < G && jr < n1t) {
@@ -365,10 +431,10 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
       for (int m = 0; m < 4; ++m) {
         // element m of the 8 loaded: 32-bit word m/2, half m%2 ; element m+4: word 2 + m/2, same half
         const uint32_t sel = (m & 1) ? 0x7632u : 0x5410u;
-        const uint32_t w0 = (m < 2) ? z[r][0].x : z[r][0].y, w1 = (m < 2) ? z[r][1].x : z[r][1].y;
-        const uint32_t w2 = (m < 2) ? z[r][2].x : z[r][2].y, w3 = (m < 2) ? z[r][3].x : z[r][3].y;
-        const uint32_t u0 = (m < 2) ? z[r][0].z : z[r][0].w, u1 = (m < 2) ? z[r][1].z : z[r][1].w;
-        const uint32_t u2 = (m < 2) ? z[r][2].z : z[r][2].w, u3 = (m < 2) ? z[r][3].z : z[r][3].w;
+        const uint32_t w0 = (m < 2) ? zt[r][0].x : zt[r][0].y, w1 = (m < 2) ? zt[r][1].x : zt[r][1].y;
+        const uint32_t w2 = (m < 2) ? zt[r][2].x : zt[r][2].y, w3 = (m < 2) ? zt[r][3].x : zt[r][3].y;
+        const uint32_t u0 = (m < 2) ? zt[r][0].z : zt[r][0].w, u1 = (m < 2) ? zt[r][1].z : zt[r][1].w;
+        const uint32_t u2 = (m < 2) ? zt[r][2].z : zt[r][2].w, u3 = (m < 2) ? zt[r][3].z : zt[r][3].w;
         mma16816(oacc[r][m], prmt(w0, w1, sel), prmt(u0, u1, sel), prmt(w2, w3, sel), prmt(u2, u3, sel), pb0, pb1);
       }
     }
@@ -379,18 +445,79 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
 #pragma unroll
         for (int sx = 0; sx < 4; ++sx) {
           const int j = jr + sx;
-          if (j < n1 && j > hole) st_global_16(vslab + (size_t)(j - 1) * D + 64 * r + 8 * gid, z[r][sx]);
+          if (j < n1 && j > hole) st_global_16(vslab + (size_t)(j - 1) * D + 64 * r + 8 * gid, zt[r][sx]);
         }
     }
-    if (it + 1 < n_iter) {
+  };
+  if constexpr (KD > 1) {
+    if (evict_one) {   // K rows behind the hole, one row up, from the registers that fed the logits
 #pragma unroll
-      for (int r = 0; r < VR; ++r)
+      for (int u = 0; u < KD; ++u) {
+        const int j0 = u * kRowsPerIter + warp * 16 + gid, j1 = j0 + 8;
 #pragma unroll
-        for (int sx = 0; sx < 4; ++sx) z[r][sx] = zn[r][sx];
+        for (int R = 0; R < QR / 2; ++R) {
+          if (j0 < n1 && j0 > hole) stg32(kslab + (size_t)(j0 - 1) * D + 64 * R + 16 * tq, xk[u][2 * R], xk[u][2 * R + 1]);
+          if (j1 < n1 && j1 > hole) stg32(kslab + (size_t)(j1 - 1) * D + 64 * R + 16 * tq, yk[u][2 * R], yk[u][2 * R + 1]);
+        }
+      }
+    }
+    // V has arrived (every thread observes every tile's barrier itself: what it reads below, and what it overwrites
+    // in global memory, has been read by the copies)
+#pragma unroll
+    for (int u = 0; u < KD; ++u)
+      if (u < n_iter) tc::mbar_wait(&vbar[u], 0, abort_flag, c.status);
+    auto v_piece = [&](int j, int piece) -> uint4* {   // 16 bytes [8 piece, +8) of row j in the swizzled tiles
+      const int u = j >> 7, r = j & 127;
+      return reinterpret_cast<uint4*>(stage + 1024 + (2 * u + (piece >> 3)) * kBoxBytes + r * 128 + (((piece & 7) ^ (r & 7)) << 4));
+    };
+    if (tid < D / 8) *v_piece(c.n_old, tid) = ld_global_16(v_new + tid * 8);   // the step's own row
+    __syncthreads();
+    if (evict_one) {   // V rows behind the hole, one row up, from shared memory; the stores drain under the MMAs below
+      const int pieces = (n1 - 1 - hole) * (D / 8);
+      for (int x = tid; x < pieces; x += kThreads) {
+        const int j = hole + 1 + x / (D / 8), pc = x % (D / 8);
+        st_global_16(vslab + (size_t)(j - 1) * D + pc * 8, *v_piece(j, pc));
+      }
+    }
+    // out^T tiles of 16 elements x heads: A = V^T (transposing ldmatrix), B = p^T of keys tb + {2tq, 2tq+1, 2tq+8, 2tq+9}
+#pragma unroll
+    for (int u = 0; u < KD; ++u) {
+      const int tb = u * kRowsPerIter + warp * 16;
+      if (u < n_iter && tb < n1t) {   // warp-uniform
+        uint32_t pb0 = 0u, pb1 = 0u;
+        if (gid < G) {
+          const float2 p0 = *reinterpret_cast<const float2*>(&s.p[gid * n1t + tb + 2 * tq]);
+          const float2 p1 = *reinterpret_cast<const float2*>(&s.p[gid * n1t + tb + 2 * tq + 8]);
+          pb0 = pack2(p0.x, p0.y);
+          pb1 = pack2(p1.x, p1.y);
+        }
+        // lane l addresses row l%8 of matrix l/8: keys tb + 8(l/16) + l%8, elements 16 dt + 8((l/8)%2) + [0, 8)
+        const int krow = tb + ((lane >> 4) << 3) + (lane & 7);
+#pragma unroll
+        for (int dt = 0; dt < D / 16; ++dt) {
+          uint32_t a0, a1, a2, a3;
+          const uint32_t addr = tc::smem_u32(v_piece(krow, 2 * dt + ((lane >> 3) & 1)));
+          asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr) : "memory");
+          mma16816(oacc[dt / 4][dt % 4], a0, a1, a2, a3, pb0, pb1);
+        }
+      }
+    }
+  } else {
+    for (int it = 0; it < n_iter; ++it) {
+      uint4 zn[VR][4];
+      if (it + 1 < n_iter) load_v(it + 1, zn);   // next iteration's rows load while this one is multiplied
+      pv_tile(it, z);
+      if (it + 1 < n_iter) {
+#pragma unroll
+        for (int r = 0; r < VR; ++r)
+#pragma unroll
+          for (int sx = 0; sx < 4; ++sx) z[r][sx] = zn[r][sx];
+      }
     }
   }
   // K rows behind the hole: one-row shift (re-read, mostly from L2: the logits pass just streamed them)
-  if (evict_one) {
+  if (KD == 1 && evict_one) {
     constexpr int PR = D / 8;                 // 16-byte pieces per row
     constexpr int RPI = kThreads / PR * 8;    // rows per iteration, 8 pieces per thread
     const int slot = tid / PR, pc = tid % PR;
@@ -419,7 +546,8 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int h = 2 * tq + (e & 1);
-        const int dd = 64 * r + 8 * gid + m + ((e & 2) ? 4 : 0);
+        // KD > 1: tile dt = 4r + m holds elements 16 dt + gid (+ 8)
+        const int dd = KD > 1 ? 16 * (4 * r + m) + gid + ((e & 2) ? 8 : 0) : 64 * r + 8 * gid + m + ((e & 2) ? 4 : 0);
         if (h < G) s.ored[(warp * G + h) * D + dd] = oacc[r][m][e];
       }
   __syncthreads();
@@ -442,21 +570,37 @@ __global__ void __launch_bounds__(NT, 512 / NT) decode_mma_kernel(CacheView c, D
   }
 }
 
-template <int D, int G, int NT, bool PLAIN>
-cudaError_t launch_nt_p(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
-  const size_t smem = decode_mma_smem_bytes(D, G, c.n_old + 1, a.target);   // sized for the larger CTA
+constexpr size_t kMaxDynamicSmem = 227 * 1024;
+// barriers + alignment slack + KD x 128 rows of V
+constexpr size_t stage_bytes(int d, int nt, int kd) { return 2048 + (size_t)kd * (nt / 32) * 16 * d * 2; }
+constexpr int kBatchTiles = 5;   // tiles per warp of the one-CTA-per-SM instance (160 registers of K rows): 640 pairs
+
+template <int D, int G, int NT, bool PLAIN, int KD>
+cudaError_t launch_nt_p(const CacheView& c, const DecodeArgs& a, cudaStream_t st, const CUtensorMap& vmap) {
+  // sized for the larger CTA; the one-CTA-per-SM instance stages all of V behind it
+  const size_t smem = decode_mma_smem_bytes(D, G, c.n_old + 1, a.target) + (KD > 1 ? stage_bytes(D, NT, KD) : 0);
   static SmemConfigured configured;
-  if (cudaError_t err = configured.ensure(decode_mma_kernel<D, G, NT, PLAIN>, smem); err != cudaSuccess) return err;
+  if (cudaError_t err = configured.ensure(decode_mma_kernel<D, G, NT, PLAIN, KD>, smem); err != cudaSuccess) return err;
   ProfileScope prof(kDecode, st);
-  const cudaError_t err = launch_dependent(decode_mma_kernel<D, G, NT, PLAIN>, dim3(c.nsamples * c.Hkv), dim3(NT), smem, st, c, a);
+  const cudaError_t err =
+      launch_dependent(decode_mma_kernel<D, G, NT, PLAIN, KD>, dim3(c.nsamples * c.Hkv), dim3(NT), smem, st, c, a, vmap);
   count_launch();
   return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 template <int D, int G, int NT>
-cudaError_t launch_nt(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
+cudaError_t launch_nt(const CacheView& c, const DecodeArgs& a, cudaStream_t st, bool one_per_sm) {
   const bool plain = c.left_pad == nullptr && c.rule == 0 && c.moved == nullptr;
-  return plain ? launch_nt_p<D, G, NT, true>(c, a, st) : launch_nt_p<D, G, NT, false>(c, a, st);
+  if constexpr (NT == 256 && D == 128) {
+    if (plain && one_per_sm && c.n_old + 1 <= kBatchTiles * (NT / 32) * 16 &&
+        decode_mma_smem_bytes(D, G, c.n_old + 1, a.target) + stage_bytes(D, NT, kBatchTiles) <= kMaxDynamicSmem) {
+      CUtensorMap vmap;
+      if (encode_slab_rows_map(&vmap, c.v_slab, D, c.n_old, c.cap, c.nsamples * c.Hkv, 128))
+        return launch_nt_p<D, G, NT, true, kBatchTiles>(c, a, st, vmap);
+    }
+  }
+  static const CUtensorMap no_map = {};   // the other instances take no tensor map
+  return plain ? launch_nt_p<D, G, NT, true, 1>(c, a, st, no_map) : launch_nt_p<D, G, NT, false, 1>(c, a, st, no_map);
 }
 
 int sm_count() {   // of the current device
@@ -477,6 +621,15 @@ int forced_threads() {   // BM_DECODE_THREADS=128|256 overrides the choice below
   return v;
 }
 
+bool batched_allowed() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = std::getenv("BM_DECODE_BATCHED");
+    v = (e == nullptr || std::atoi(e) != 0) ? 1 : 0;
+  }
+  return v != 0;
+}
+
 template <int D, int G>
 cudaError_t launch_t(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
   const int f = forced_threads();
@@ -485,7 +638,10 @@ cudaError_t launch_t(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
   // caches: 0.96 against 0.69)
   const bool four_fit = c.n_old + 1 <= 1536 && smem_layout(nullptr, D, G, c.n_old + 1, 4, nullptr) <= 56 * 1024;
   const bool small_ctas = f == 128 || (f != 256 && four_fit && c.nsamples * c.Hkv > 2 * sm_count());
-  return small_ctas ? launch_nt<D, G, 128>(c, a, st) : launch_nt<D, G, 256>(c, a, st);
+  // a grid that leaves every CTA an SM of its own: the instance that keeps K in registers (BM_DECODE_BATCHED=0
+  // turns it off, a tuning aid)
+  const bool one_per_sm = c.nsamples * c.Hkv <= sm_count() && batched_allowed();
+  return small_ctas ? launch_nt<D, G, 128>(c, a, st, false) : launch_nt<D, G, 256>(c, a, st, one_per_sm);
 }
 
 template <int D>

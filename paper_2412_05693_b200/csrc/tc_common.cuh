@@ -7,6 +7,9 @@
 #include <stdint.h>
 
 namespace bm {
+// (attn_tc.cu) tensor map over the first `rows` rows of every cache of a bf16 slab: tiles of box_rows x 64 elements,
+// 128-byte swizzle, rows past `rows` read as zeros; false when the driver's encoder is unavailable
+bool encode_slab_rows_map(CUtensorMap* m, const void* slab, int d, int rows, int cap, int units, int box_rows);
 namespace tc {
 
 constexpr int kErrTimeout = 6;            // BM_ERR_TIMEOUT
