@@ -250,7 +250,8 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
   // first V tile and the old sum_weights start loading now; they are needed only after the softmax
   uint4 z[VR][4];
   // KD > 1: all of V starts on its way into shared memory now, as TMA tiles of 128 rows x 64 elements (128-byte
-  // swizzle; rows past n_old arrive as zeros), one mbarrier per 128 rows.  The copies stream while the softmax
+  // swizzle; rows past n_old arrive as zeros), one mbarrier per 128 rows; the tiles of each half of the row lie
+  // one behind the other, so that each half is one array of 128-byte rows.  The copies stream while the softmax
   // phases run and pass by the register file, whose write-back path those phases need (the same rows prefetched
   // into registers made the phases longer by the time the loads took; per-thread cp.async stalled at issue).
   const uint32_t stage0 = (tc::smem_u32(smem_raw) + (uint32_t)smem_layout(nullptr, D, G, n1, kWarps, nullptr) + 1023u) & ~1023u;
@@ -264,8 +265,8 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
       for (int u = 0; u < KD; ++u)
         if (u < n_iter) {
           tc::mbar_expect_tx(&vbar[u], 2 * kBoxBytes);
-          tc::tma_load_3d(stage + 1024 + (2 * u) * kBoxBytes, &vmap, 0, u * 128, unit, &vbar[u]);
-          tc::tma_load_3d(stage + 1024 + (2 * u + 1) * kBoxBytes, &vmap, 64, u * 128, unit, &vbar[u]);
+          tc::tma_load_3d(stage + 1024 + u * kBoxBytes, &vmap, 0, u * 128, unit, &vbar[u]);
+          tc::tma_load_3d(stage + 1024 + (KD + u) * kBoxBytes, &vmap, 64, u * 128, unit, &vbar[u]);
         }
     }
   } else {
@@ -467,16 +468,29 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
     for (int u = 0; u < KD; ++u)
       if (u < n_iter) tc::mbar_wait(&vbar[u], 0, abort_flag, c.status);
     auto v_piece = [&](int j, int piece) -> uint4* {   // 16 bytes [8 piece, +8) of row j in the swizzled tiles
-      const int u = j >> 7, r = j & 127;
-      return reinterpret_cast<uint4*>(stage + 1024 + (2 * u + (piece >> 3)) * kBoxBytes + r * 128 + (((piece & 7) ^ (r & 7)) << 4));
+      return reinterpret_cast<uint4*>(stage + 1024 + (piece >> 3) * (KD * kBoxBytes) + j * 128 + (((piece & 7) ^ (j & 7)) << 4));
     };
-    if (tid < D / 8) *v_piece(c.n_old, tid) = ld_global_16(v_new + tid * 8);   // the step's own row
+    if (tid < D / 8) {   // the step's own row
+      *v_piece(c.n_old, tid) = ld_global_16(v_new + tid * 8);
+      tc::fence_async_smem();   // the TMA stores below read it
+    }
     __syncthreads();
-    if (evict_one) {   // V rows behind the hole, one row up, from shared memory; the stores drain under the MMAs below
-      const int pieces = (n1 - 1 - hole) * (D / 8);
-      for (int x = tid; x < pieces; x += kThreads) {
-        const int j = hole + 1 + x / (D / 8), pc = x % (D / 8);
+    if (evict_one) {
+      // V rows behind the hole, one row up, from shared memory: up to the next multiple of 8 rows (the swizzle's
+      // period) by plain stores, the rest as TMA tiles of 128 rows written one row higher than they were read
+      // (rows past n_old - 1 are clipped by the map); they drain under the MMAs below
+      const int r8 = (hole + 8) & ~7;
+      const int pieces = (min(r8, n1) - 1 - hole) * (D / 8);
+      if (tid < pieces) {
+        const int j = hole + 1 + tid / (D / 8), pc = tid % (D / 8);
         st_global_16(vslab + (size_t)(j - 1) * D + pc * 8, *v_piece(j, pc));
+      }
+      if (tid == 0) {
+        for (int r0 = r8; r0 < n1; r0 += 128) {
+          tc::tma_store_3d(&vmap, stage + 1024 + r0 * 128, 0, r0 - 1, unit);
+          tc::tma_store_3d(&vmap, stage + 1024 + KD * kBoxBytes + r0 * 128, 64, r0 - 1, unit);
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
       }
     }
     // out^T tiles of 16 elements x heads: A = V^T (transposing ldmatrix), B = p^T of keys tb + {2tq, 2tq+1, 2tq+8, 2tq+9}
@@ -559,6 +573,9 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
     op[t] = __float2bfloat16_rn(tot);
   }
 
+  if constexpr (KD > 1) {   // the TMA stores have read their rows out of shared memory
+    if (tid == 0 && evict_one) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+  }
   if (evict_general) {
     __syncthreads();
     CacheView cv = c;

@@ -67,6 +67,10 @@ __device__ __forceinline__ void tma_store_5d(const CUtensorMap* map, const void*
   asm volatile("cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4, %5}], [%6];"
                ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(smem_u32(src)) : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(src)) : "memory");
+}
 // Commits the stores issued so far and waits until their shared-memory source has been read (the global
 // writes themselves complete asynchronously; kernel completion makes them visible).
 __device__ __forceinline__ void tma_store_commit_and_wait() {
