@@ -478,15 +478,21 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
     if (evict_one) {
       // V rows behind the hole, one row up, from shared memory: up to the next multiple of 8 rows (the swizzle's
       // period) by plain stores, the rest as TMA tiles of 128 rows written one row higher than they were read
-      // (rows past n_old - 1 are clipped by the map); they drain under the MMAs below
+      // (rows past n_old - 1 are clipped by the map); they drain under the MMAs below.  A tile that would read past
+      // the staged rows is not stored: the rows from r_tail on (fewer than 128) leave by plain stores as well.
       const int r8 = (hole + 8) & ~7;
+      const int r_tail = r8 > (KD - 1) * 128 ? r8 : r8 + 128 * (((KD - 1) * 128 - r8) / 128 + 1);
       const int pieces = (min(r8, n1) - 1 - hole) * (D / 8);
       if (tid < pieces) {
         const int j = hole + 1 + tid / (D / 8), pc = tid % (D / 8);
         st_global_16(vslab + (size_t)(j - 1) * D + pc * 8, *v_piece(j, pc));
       }
+      for (int x = tid; x < (n1 - r_tail) * (D / 8); x += kThreads) {
+        const int j = r_tail + x / (D / 8), pc = x % (D / 8);
+        st_global_16(vslab + (size_t)(j - 1) * D + pc * 8, *v_piece(j, pc));
+      }
       if (tid == 0) {
-        for (int r0 = r8; r0 < n1; r0 += 128) {
+        for (int r0 = r8; r0 < min(n1, r_tail); r0 += 128) {
           tc::tma_store_3d(&vmap, stage + 1024 + r0 * 128, 0, r0 - 1, unit);
           tc::tma_store_3d(&vmap, stage + 1024 + KD * kBoxBytes + r0 * 128, 64, r0 - 1, unit);
         }

@@ -197,6 +197,16 @@ def test_decode_with_more_caches_than_two_ctas_per_sm(g):
     assert st["evictions"] >= len(units) * 10
 
 
+@pytest.mark.parametrize("K,g", [(511, 4), (512, 1), (600, 4), (639, 2), (640, 4)])
+def test_decode_with_one_cache_per_sm(K, g):
+    # few caches of at most 640 pairs: the decode kernel's instance that keeps K in registers and stages V by TMA
+    # (rows behind the pair that leaves move up as TMA tiles, their first rows and a tail past the staged rows by
+    # plain stores); 641 pairs fall back to the other instance
+    wl = tiny("one_per_sm", b=3, Hq=2 * g, Hkv=2, s=K + 140, B=128, K=K, steps=14, dtype="bf16", d=128)
+    st = run_lockstep(wl, all_units(wl), check_rows_every=1)
+    assert st["evictions"] >= 6 * 14
+
+
 # ------------------------------------------------------------------ the rules of Sec. 2 on the same kernels
 @pytest.mark.parametrize("rule", ["sum_recent", "current_query"])
 @pytest.mark.parametrize("dtype,d,Hq,Hkv", [("bf16", 128, 8, 2), ("f32", 64, 4, 4)])
