@@ -102,8 +102,8 @@ __device__ __forceinline__ void stg32(__nv_bfloat16* p, const uint4& lo, const u
                :: "l"(p), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
 }
 
-// PLAIN: no left padding, the paper's own eviction rule, no counting of moved rows -- the instance the common case
-// runs, free of those branches.
+// PLAIN: no left padding and the paper's own eviction rule -- the instance the common case runs, free of those
+// branches.
 // KD: 1 = every warp keeps one tile of rows in flight beyond the one it multiplies (fits the register budget of two
 // or four CTAs per SM).  KD > 1 = one CTA per SM with the whole register file, for caches of at most KD tiles per
 // warp in grids of at most one CTA per SM: all of K is loaded at once and stays in registers until the pair that
@@ -395,7 +395,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
       if (oa < best_ave || (oa == best_ave && oj > best_j)) { best_ave = oa; best_j = oj; }
     }
     hole = best_j;
-    if (!PLAIN && c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)(n1 - 1 - hole));
+    if (c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)(n1 - 1 - hole));
     // sum_weights / kv_ids in their final places: rows behind the hole move up by one
     for (int j = tid; j < n1; j += kThreads) {
       if (j < hole) c.sum_weights[base + j] = s.score[j];
@@ -613,7 +613,7 @@ cudaError_t launch_nt_p(const CacheView& c, const DecodeArgs& a, cudaStream_t st
 
 template <int D, int G, int NT>
 cudaError_t launch_nt(const CacheView& c, const DecodeArgs& a, cudaStream_t st, bool one_per_sm) {
-  const bool plain = c.left_pad == nullptr && c.rule == 0 && c.moved == nullptr;
+  const bool plain = c.left_pad == nullptr && c.rule == 0;
   if constexpr (NT == 256 && D == 128) {
     if (plain && one_per_sm && c.n_old + 1 <= kBatchTiles * (NT / 32) * 16 &&
         decode_mma_smem_bytes(D, G, c.n_old + 1, a.target) + stage_bytes(D, NT, kBatchTiles) <= kMaxDynamicSmem) {
