@@ -117,6 +117,42 @@ def arm_calls(wl: Workload, arm: str, kv_bar: int | None = None, p: int = 64):
     return calls
 
 
+GRAPH_DECODE_INPUT_BYTES = 256 << 20
+
+
+def _decode_phase_as_graph(cache, inp, calls, layer, n, out_dec):
+    """Captures the calls of a decode phase (decode steps and the cuts between them) on the whole batch in one CUDA
+    graph, replays it once between two events; returns (ms, cached pairs at the end, rows read by the decode steps)."""
+    ins = []
+    for kind, pos0, I, arg in calls:
+        if kind == "decode":
+            q, k, v = inp.block(layer, pos0, 1)
+            ins.append((q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous()))
+    rows = 0
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        it = iter(ins)
+        for kind, pos0, I, arg in calls:
+            if kind == "decode":
+                q, k, v = next(it)
+                cache.decode_step(q, k, v, out=out_dec[:q.shape[0]], evict_to=arg, layer=layer)
+                rows += n + 1
+                n = n + 1 if arg < 0 else min(n + 1, arg)
+            else:
+                assert kind in ("evict", "recent"), kind
+                (cache.evict if kind == "evict" else cache.keep_most_recent)(arg, layer=layer)
+                n = min(n, arg)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record()
+        graph.replay()
+        e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1), n, rows
+
+
 class Timer:
     def __init__(self):
         self.pairs = []
@@ -157,11 +193,20 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
     out_dec = torch.empty(micro_dec, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
     calls = arm_calls(wl, arm, kv_bar, p)
     pairs = dec_rows = 0
+    # a small batch decodes in steps of a few tens of microseconds, which eager launches from Python cannot feed: its
+    # decode phase (every call from the first decode step on) is captured once in a CUDA graph and replayed
+    e_in = (wl.Hq + 2 * wl.Hkv) * wl.d * wl.elem_bytes
+    graph_decode = batch <= micro_dec and wl.steps * batch * e_in <= GRAPH_DECODE_INPUT_BYTES
     for layer in layers:
         n, in_decode, pending = 0, False, 0
-        for kind, pos0, I, arg in calls:
+        for ci, (kind, pos0, I, arg) in enumerate(calls):
             if kind == "decode" and not in_decode:
                 moved_pre = cache.moved_rows(reset=True)
+                if graph_decode:
+                    ms, n, rows = _decode_phase_as_graph(cache, inp, calls[ci:], layer, n, out_dec)
+                    ms_dec += ms
+                    dec_rows += rows
+                    break
             in_decode = in_decode or kind == "decode"
             timer = t_dec if in_decode else t_pre
             if kind == "prefill":
@@ -233,7 +278,8 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
         "note": "prefill = every call before the first decode step (attention, score pass, evictions; the whole call, "
                 "not the forward kernel alone); decode = every call from the first decode step on; decode bytes "
                 "exclude compaction moves; every prefill call and every decode step (all its sample ranges) timed with its own "
-                "CUDA events",
+                "CUDA events" + ("; the decode phase of this small batch is one CUDA graph, replayed once between two events"
+                                 if graph_decode else ""),
     }
     if arm in ("alg1", "ed"):
         res["kv_bar"] = kv_bar
