@@ -39,7 +39,10 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
   const int R = a.I * a.g;
   const int qpt = kTileM / a.g;                  // inputs (positions) covered by the row tile
   const int t_old = (a.n_old + kTileN - 1) / kTileN;
-  const int row0 = blockIdx.x * kTileM, i0 = blockIdx.x * qpt;
+  // row tiles are handed out last first: a later tile sees more of the block's own keys, and the longest CTAs of a
+  // cache should not be the ones that start last
+  const int rt = gridDim.x - 1 - blockIdx.x;
+  const int row0 = rt * kTileM, i0 = rt * qpt;
   const int T = t_old + min(a.I - 1, i0 + qpt - 1) / kTileN + 1;   // cached-key tiles + block-key tiles up to the last input
 
   auto load_kv = [&](int e) {   // ring entry e: K_j for even e, V_j for odd e, j = e / 2
