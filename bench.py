@@ -47,6 +47,9 @@ def parse_args():
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
     ap.add_argument("--rule", default="average", choices=["average", "sum_recent", "current_query"],
                     help="eviction rule: the paper's average attention, or one of the two rules of Sec. 2")
+    ap.add_argument("--compaction", default="stable", choices=["stable", "fill"],
+                    help="stable: a cache's rows stay in position order (rows behind a pair that leaves move up); "
+                         "fill: unordered rows, pairs that stay never move (same kept sets and outputs)")
     ap.add_argument("--ragged", action="store_true",
                     help="left-padded samples: seeded padding counts in [0, s/2] (sample 0 unpadded); launches eagerly")
     return ap.parse_args()
@@ -230,7 +233,8 @@ def main():
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     calls = schedule(wl)
-    cfg = make_config(wl, device=local_rank, rule=args.rule)
+    cfg = make_config(wl, device=local_rank, rule=args.rule, compaction=args.compaction)
+    cfg_now = [cfg]      # the configuration one_step() builds its cache with
     stream = torch.cuda.current_stream()
 
     # ---- inputs resident in HBM (layer 0's stream is reused for every layer: layers are independent)
@@ -256,7 +260,7 @@ def main():
         args.no_graph = True     # the padding counts are copied from pageable host memory at the start of a step
 
     def one_step(host_bufs=None, with_decode=True, moved=None):
-        cache = bm.BatchMaxCache(cfg, arena=arena, workspace=workspace)
+        cache = bm.BatchMaxCache(cfg_now[0], arena=arena, workspace=workspace)
         if pads is not None:
             cache.set_left_pad(pads)
         if moved is not None:                 # count the rows the compactions move, prefill and decode apart
@@ -325,6 +329,16 @@ def main():
     ms_step = timed(args.warmup, args.steps, use_graph=not args.no_graph)
     # the same step without its decode calls: the difference is the decode steps' time inside the timed region
     ms_prefill_only = timed(1, args.steps, use_graph=not args.no_graph, with_decode=False) if wl.steps > 0 else ms_step
+    # the same step on unordered caches (pairs that stay never move; same kept sets and outputs), as a variant line
+    variants = {}
+    if args.compaction == "stable" and args.rule == "average" and not args.ragged:
+        cfg_now[0] = make_config(wl, device=local_rank, rule=args.rule, compaction="fill")
+        ms_fill = timed(args.warmup, args.steps, use_graph=not args.no_graph)
+        cfg_now[0] = cfg
+        variants["compaction_fill"] = {
+            "ms_per_step": ms_fill, "value": whole_job_value(workload_tokens(wl), world, ms_fill), "unit": "tokens/s",
+            "note": "BM_COMPACT_FILL: a cache's rows are an unordered set, the pairs that arrive take the rows that "
+                    "were freed; the headline value is measured with rows kept in position order"}
     launches = launches_per_step * args.steps
     clocks = sampler.stop() if rank == 0 else None
     tokens = workload_tokens(wl)
@@ -410,12 +424,14 @@ def main():
                 "config": cfg_dict(wl, {"parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                                         "prefill_path": "tcgen05" if bm.last_prefill_path() == 1 else "simt-fp32",
                                         "launch": "eager" if args.no_graph else "one CUDA graph per step, replayed",
-                                        "rule": args.rule,
+                                        "rule": args.rule, "compaction": args.compaction,
                                         "left_pad": "none" if pads is None else
                                         f"seeded, {sum(pads)} of {wl.b * wl.s} prompt positions are padding"}),
                 "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": int(launches),
                 "clocks": clocks, "prefill_useful_tflop_per_step": 4.0 * wl.d * ppairs / 1e12}
         line.update(extra)
+        if variants:
+            line["variants"] = variants
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

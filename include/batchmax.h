@@ -64,6 +64,16 @@ typedef enum { BM_F32 = 0, BM_BF16 = 1 } bm_dtype_t;
  * Ties keep the lower position under every rule. */
 typedef enum { BM_RULE_AVERAGE = 0, BM_RULE_SUM_RECENT = 1, BM_RULE_CURRENT_QUERY = 2 } bm_rule_t;
 
+/* What "remove pairs" does to the rows of a cache.  Attention, the scores and the kept sets do not depend on the
+ * order of a cache's rows; only the work of removing does.
+ *   BM_COMPACT_STABLE: rows stay in ascending kv_ids order; the rows behind a pair that leaves move up.
+ *   BM_COMPACT_FILL:   rows are an unordered set: a pair that stays never moves, the pairs that arrive (the block's
+ *                      kept pairs, the decode step's pair) take the rows that were freed.  Kept sets, sum_weights and
+ *                      outputs are the same as under BM_COMPACT_STABLE (ties still keep the lower position, decided
+ *                      on kv_ids); bm_cache_export returns the rows in storage order.  Only with BM_RULE_AVERAGE;
+ *                      bm_cache_set_left_pad with a non-zero count and bm_keep_most_recent return BM_ERR_INVALID. */
+typedef enum { BM_COMPACT_STABLE = 0, BM_COMPACT_FILL = 1 } bm_compaction_t;
+
 /* Problem statement: Algorithm 1's inputs (\overline{|kv|}, p) generalised as (K, growth), plus the
  * attention shape.  All sizes in elements. */
 typedef struct {
@@ -80,6 +90,7 @@ typedef struct {
   int32_t device;           /* CUDA device ordinal                                            */
   int32_t max_call_samples; /* largest nsamples of any call (sizes the workspace); 0 -> batch */
   int32_t rule;             /* bm_rule_t: what pairs are ranked by at an eviction; 0 = the paper's  */
+  int32_t compaction;       /* bm_compaction_t: 0 = rows stay in position order                     */
 } bm_config_t;
 
 /* ---- cache layout, allocator and memory model (Sec. 1: batch size under a fixed memory budget) ----

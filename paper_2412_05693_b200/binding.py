@@ -29,7 +29,7 @@ class bm_config_t(C.Structure):
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("kv_max", C.c_int32),
                 ("block_max", C.c_int32), ("growth", C.c_int32), ("dtype", C.c_int32),
                 ("softmax_scale", C.c_float), ("device", C.c_int32), ("max_call_samples", C.c_int32),
-                ("rule", C.c_int32)]
+                ("rule", C.c_int32), ("compaction", C.c_int32)]
 
 
 _lib = None
@@ -105,12 +105,14 @@ class Config:
     device: int = 0
     max_call_samples: int = 0
     rule: str = "average"        # "average" (the paper's) | "sum_recent" | "current_query"
+    compaction: str = "stable"   # "stable": rows stay in position order | "fill": unordered, kept pairs never move
 
     def c(self) -> bm_config_t:
         return bm_config_t(self.batch, self.n_layers, self.n_q_heads, self.n_kv_heads, self.head_dim, self.kv_max,
                            self.block_max, self.growth, BM_BF16 if self.dtype == "bf16" else BM_F32,
                            self.softmax_scale, self.device, self.max_call_samples,
-                           {"average": 0, "sum_recent": 1, "current_query": 2}[self.rule])
+                           {"average": 0, "sum_recent": 1, "current_query": 2}[self.rule],
+                           {"stable": 0, "fill": 1}[self.compaction])
 
     @property
     def cap(self) -> int:

@@ -66,6 +66,8 @@ bool config_ok(const bm_config_t* c, bool need_batch) {
   if (!(c->softmax_scale >= 0.f) || std::isinf(c->softmax_scale)) return false;
   if (c->device < 0 || c->max_call_samples < 0) return false;
   if (c->rule < 0 || c->rule > 2) return false;
+  if (c->compaction < 0 || c->compaction > 1) return false;
+  if (c->compaction == BM_COMPACT_FILL && c->rule != BM_RULE_AVERAGE) return false;
   if ((long long)c->kv_max + c->growth > (1 << 24)) return false;
   return true;
 }
@@ -186,6 +188,7 @@ CacheView make_view(const bm_cache* c, int layer, int sample0, int nsamples, int
   v.status = c->status;
   v.left_pad = (c->has_pad && with_pad) ? c->left_pad + sample0 : nullptr;
   v.rule = c->cfg.rule;
+  v.fill = c->cfg.compaction == BM_COMPACT_FILL ? 1 : 0;
   v.moved = c->count_moves ? reinterpret_cast<unsigned long long*>(c->status + 16) : nullptr;
   return v;
 }
@@ -404,6 +407,7 @@ bm_status_t bm_evict(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsam
 
 bm_status_t bm_keep_most_recent(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, int32_t keep,
                                 void* cuda_stream) {
+  if (c != nullptr && c->cfg.compaction == BM_COMPACT_FILL) return BM_ERR_INVALID;   // the rule ranks rows by their order
   return evict_cached(c, layer, sample0, nsamples, keep, true, cuda_stream);
 }
 
@@ -547,6 +551,7 @@ bm_status_t bm_cache_set_left_pad(bm_cache_t* c, const int32_t* pads, void* cuda
       if (pads[s] < 0) return BM_ERR_INVALID;
       any = any || pads[s] > 0;
     }
+  if (any && c->cfg.compaction == BM_COMPACT_FILL) return BM_ERR_INVALID;   // padding is a prefix of an ordered cache
   c->has_pad = any;
   if (!any) return BM_OK;
   c->pad_host.assign(pads, pads + c->cfg.batch);

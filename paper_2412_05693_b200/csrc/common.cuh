@@ -21,6 +21,7 @@ struct CacheView {
   const int32_t* left_pad;  // [nsamples] padding positions at the start of each sample of the range, or null
   unsigned long long* moved;  // [16] counters of rows moved by compactions (unit & 15), or null when not counting
   int32_t rule;             // 0 average attention (Sec. 3.2), 1 sum + window of recent pairs, 2 current query (Sec. 2)
+  int32_t fill;             // 1: unordered cache -- pairs that stay never move, new pairs fill the freed rows
 };
 
 // Left padding (Sec. 3): positions below the sample's count are padding.  A padding pair is masked for every

@@ -78,8 +78,9 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
   const size_t base = (size_t)unit * c.cap;
   T* kslab = reinterpret_cast<T*>(c.k_slab) + base * D;
   T* vslab = reinterpret_cast<T*>(c.v_slab) + base * D;
-  const bool evict_one = (a.target == n1 - 1);
-  const bool evict_general = (a.target >= 0 && a.target < n1 - 1);
+  // (an unordered cache takes the general path for every cut: there the new pair fills the freed row)
+  const bool evict_one = (a.target == n1 - 1) && !c.fill;
+  const bool evict_general = (a.target >= 0 && a.target < n1 && !evict_one);
   // left-padded sample: padding pairs are masked and leave first; a query at a padding position (not a real
   // decode step) gets a zero output and no weights
   const int pad = sample_left_pad(c, smp);
@@ -356,7 +357,7 @@ cudaError_t launch_g(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
 
 size_t decode_smem_bytes(int d, int g, int n_rows, int target) {
   const size_t attn = dec_smem_layout(nullptr, d, g, n_rows, nullptr);
-  const size_t ev = (target >= 0 && target < n_rows - 1) ? evict_smem_bytes(n_rows, target) : 0;
+  const size_t ev = (target >= 0 && target < n_rows) ? evict_smem_bytes(n_rows, target) : 0;
   return attn > ev ? attn : ev;
 }
 

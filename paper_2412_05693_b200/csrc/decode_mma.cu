@@ -40,7 +40,7 @@ struct Smem {
   float* score;   // [n1t]
   int32_t* id;    // [n1t]
   float* wred;    // [2][G][warps]
-  float* best;    // [2][warps]
+  float* best;    // [3][warps]
   float* ored;    // [warps][G][D]
 };
 
@@ -49,7 +49,7 @@ __host__ __device__ inline size_t smem_layout(unsigned char* base, int d, int g,
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) & ~size_t(15); return o; };
   const size_t op = take(4 * (size_t)g * n1t), os = take(4 * n1t), oi = take(4 * n1t);
-  const size_t ow = take(4 * 2 * (size_t)g * kWarps), ob = take(4 * 2 * kWarps), oo = take(4 * (size_t)kWarps * g * d);
+  const size_t ow = take(4 * 2 * (size_t)g * kWarps), ob = take(4 * 3 * kWarps), oo = take(4 * (size_t)kWarps * g * d);
   if (s != nullptr) {
     s->p = reinterpret_cast<float*>(base + op);
     s->score = reinterpret_cast<float*>(base + os);
@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
 
   // ---- normalise, sum_weights += attn_weights (heads added in a fixed order), candidate for eviction
   float best_ave = INFINITY;
-  int best_j = -1;
+  int best_j = -1, best_id = -1;
   for (int j = tid, u = 0; j < n1t; j += kThreads, ++u) {
     if (j >= n1) {
 #pragma unroll
@@ -371,7 +371,8 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
       // fast division: the IEEE routine takes a slow path for the tiny sums of long-evicted histories (4 % of the step)
       else if (rule == 0) ave = __fdividef(sw, (float)G * (float)(a.pos + 1 - s.id[j]));
       else ave = (rule == 1 && j >= n1 - a.target / 2) ? INFINITY : sw;
-      if (ave <= best_ave) { best_ave = ave; best_j = j; }   // j ascends: ties move to the higher position
+      // ties: the higher position leaves (kv_ids, not rows: the rows of an unordered cache are in no order)
+      if (ave < best_ave || (ave == best_ave && s.id[j] > best_id)) { best_ave = ave; best_j = j; best_id = s.id[j]; }
     } else {
       c.sum_weights[base + j] = sw;
     }
@@ -381,25 +382,39 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
       const float oa = __shfl_xor_sync(0xffffffffu, best_ave, off);
-      const int oj = __shfl_xor_sync(0xffffffffu, best_j, off);
-      if (oa < best_ave || (oa == best_ave && oj > best_j)) { best_ave = oa; best_j = oj; }
+      const int oj = __shfl_xor_sync(0xffffffffu, best_j, off), oi = __shfl_xor_sync(0xffffffffu, best_id, off);
+      if (oa < best_ave || (oa == best_ave && oi > best_id)) { best_ave = oa; best_j = oj; best_id = oi; }
     }
-    if (lane == 0) { s.best[warp] = best_ave; reinterpret_cast<int*>(s.best)[kWarps + warp] = best_j; }
+    if (lane == 0) {
+      s.best[warp] = best_ave;
+      reinterpret_cast<int*>(s.best)[kWarps + warp] = best_j;
+      reinterpret_cast<int*>(s.best)[2 * kWarps + warp] = best_id;
+    }
     __syncthreads();
     best_ave = s.best[0];
     best_j = reinterpret_cast<int*>(s.best)[kWarps];
+    best_id = reinterpret_cast<int*>(s.best)[2 * kWarps];
 #pragma unroll
     for (int w = 1; w < kWarps; ++w) {
       const float oa = s.best[w];
-      const int oj = reinterpret_cast<int*>(s.best)[kWarps + w];
-      if (oa < best_ave || (oa == best_ave && oj > best_j)) { best_ave = oa; best_j = oj; }
+      const int oj = reinterpret_cast<int*>(s.best)[kWarps + w], oi = reinterpret_cast<int*>(s.best)[2 * kWarps + w];
+      if (oa < best_ave || (oa == best_ave && oi > best_id)) { best_ave = oa; best_j = oj; best_id = oi; }
     }
     hole = best_j;
-    if (c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)(n1 - 1 - hole));
-    // sum_weights / kv_ids in their final places: rows behind the hole move up by one
-    for (int j = tid; j < n1; j += kThreads) {
-      if (j < hole) c.sum_weights[base + j] = s.score[j];
-      else if (j > hole) { c.sum_weights[base + j - 1] = s.score[j]; c.kv_ids[base + j - 1] = s.id[j]; }
+    if (c.fill) {
+      // unordered cache: every pair stays where it is and the step's own pair takes the row of the pair that leaves
+      if (c.moved != nullptr && tid == 0 && hole < c.n_old) atomicAdd(&c.moved[unit & 15], 1ull);
+      for (int j = tid; j < c.n_old; j += kThreads) {
+        if (j != hole) c.sum_weights[base + j] = s.score[j];
+        else { c.sum_weights[base + j] = s.score[c.n_old]; c.kv_ids[base + j] = a.pos; }
+      }
+    } else {
+      if (c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)(n1 - 1 - hole));
+      // sum_weights / kv_ids in their final places: rows behind the hole move up by one
+      for (int j = tid; j < n1; j += kThreads) {
+        if (j < hole) c.sum_weights[base + j] = s.score[j];
+        else if (j > hole) { c.sum_weights[base + j - 1] = s.score[j]; c.kv_ids[base + j - 1] = s.id[j]; }
+      }
     }
   } else {
     if (tid == 0) c.kv_ids[base + c.n_old] = a.pos;
@@ -439,7 +454,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
         mma16816(oacc[r][m], prmt(w0, w1, sel), prmt(u0, u1, sel), prmt(w2, w3, sel), prmt(u2, u3, sel), pb0, pb1);
       }
     }
-    if (evict_one && (it + 1) * kRowsPerIter > hole) {   // uniform over the CTA
+    if (evict_one && !c.fill && (it + 1) * kRowsPerIter > hole) {   // uniform over the CTA
       __syncthreads();                                   // every load of rows < (it+1)*kRowsPerIter has completed
 #pragma unroll
       for (int r = 0; r < VR; ++r)
@@ -451,7 +466,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
     }
   };
   if constexpr (KD > 1) {
-    if (evict_one) {   // K rows behind the hole, one row up, from the registers that fed the logits
+    if (evict_one && !c.fill) {   // K rows behind the hole, one row up, from the registers that fed the logits
 #pragma unroll
       for (int u = 0; u < KD; ++u) {
         const int j0 = u * kRowsPerIter + warp * 16 + gid, j1 = j0 + 8;
@@ -475,7 +490,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
       tc::fence_async_smem();   // the TMA stores below read it
     }
     __syncthreads();
-    if (evict_one) {
+    if (evict_one && !c.fill) {
       // V rows behind the hole, one row up, from shared memory: up to the next multiple of 8 rows (the swizzle's
       // period) by plain stores, the rest as TMA tiles of 128 rows written one row higher than they were read
       // (rows past n_old - 1 are clipped by the map); they drain under the MMAs below.  A tile that would read past
@@ -537,7 +552,15 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
     }
   }
   // K rows behind the hole: one-row shift (re-read, mostly from L2: the logits pass just streamed them)
-  if (KD == 1 && evict_one) {
+  if (evict_one && c.fill) {
+    // unordered cache: the step's own pair takes the row of the pair that leaves (every read of that row is over)
+    __syncthreads();
+    if (hole < c.n_old && tid < 2 * (D / 8)) {
+      const int pc = tid % (D / 8);
+      T* dst = (tid < D / 8 ? kslab : vslab) + (size_t)hole * D + pc * 8;
+      st_global_16(dst, ld_global_16((tid < D / 8 ? k_new : v_new) + pc * 8));
+    }
+  } else if (KD == 1 && evict_one) {
     constexpr int PR = D / 8;                 // 16-byte pieces per row
     constexpr int RPI = kThreads / PR * 8;    // rows per iteration, 8 pieces per thread
     const int slot = tid / PR, pc = tid % PR;
@@ -580,7 +603,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
   }
 
   if constexpr (KD > 1) {   // the TMA stores have read their rows out of shared memory
-    if (tid == 0 && evict_one) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+    if (tid == 0 && evict_one && !c.fill) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
   }
   if (evict_general) {
     __syncthreads();

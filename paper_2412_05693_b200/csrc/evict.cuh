@@ -14,7 +14,8 @@ namespace bm {
 struct EvictSmem {
   float* score;    // [n_cand]
   int32_t* id;     // [n_cand]
-  int32_t* src;    // [target]   candidate index that lands in row r
+  int32_t* src;    // [target]   candidate index that lands in row r (fill mode: k-th candidate that has to move)
+  int32_t* dst;    // [target]   fill mode: row the k-th moving candidate lands in
   uint32_t* hist;  // [256]
   int32_t* misc;   // [8]
   int32_t* wsum;   // [64]
@@ -24,12 +25,14 @@ __host__ __device__ inline size_t evict_smem_layout(unsigned char* base, int n_c
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) & ~size_t(15); return o; };
   size_t o_score = take(sizeof(float) * n_cand), o_id = take(sizeof(int32_t) * n_cand);
-  size_t o_src = take(sizeof(int32_t) * (target > 0 ? target : 1)), o_hist = take(sizeof(uint32_t) * 256);
+  size_t o_src = take(sizeof(int32_t) * (target > 0 ? target : 1)), o_dst = take(sizeof(int32_t) * (target > 0 ? target : 1));
+  size_t o_hist = take(sizeof(uint32_t) * 256);
   size_t o_misc = take(sizeof(int32_t) * 8), o_wsum = take(sizeof(int32_t) * 64);
   if (s != nullptr) {
     s->score = reinterpret_cast<float*>(base + o_score);
     s->id = reinterpret_cast<int32_t*>(base + o_id);
     s->src = reinterpret_cast<int32_t*>(base + o_src);
+    s->dst = reinterpret_cast<int32_t*>(base + o_dst);
     s->hist = reinterpret_cast<uint32_t*>(base + o_hist);
     s->misc = reinterpret_cast<int32_t*>(base + o_misc);
     s->wsum = reinterpret_cast<int32_t*>(base + o_wsum);
@@ -82,23 +85,17 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
     return s.id[j] < pad ? 0u : max(b, 1u);   // padding pairs rank below every real pair (left-padded samples)
   };
 
-  if (target >= n_c) {
-    for (int r = tid; r < n_c; r += NT) s.src[r] = r;
-    __syncthreads();
-  } else if (e.recent) {  // Algorithm 3's rule: the most recent pairs stay, whatever their weights
-    for (int r = tid; r < target; r += NT) s.src[r] = n_c - target + r;
-    __syncthreads();
-  } else {
-    // ---- radix select: bit pattern `thr` of the target-th largest ave, and how many equal to it to keep
+  // Radix select over the candidates `key_of` admits: the key of the need-th largest, and how many candidates equal
+  // to that key belong to the `need` largest.  Four passes of 8 bits, histogram in shared memory.
+  auto radix_kth_largest = [&](auto key_of, int need, uint32_t& out_key, int& out_need_eq) {
     uint32_t prefix = 0, mask = 0;
-    int need = target;
     for (int pass = 0; pass < 4; ++pass) {
       const int shift = 24 - 8 * pass;
       for (int t = tid; t < 256; t += NT) s.hist[t] = 0;
       __syncthreads();
       for (int j = tid; j < n_c; j += NT) {
-        const uint32_t b = ave_bits(j);
-        if ((b & mask) == prefix) atomicAdd(&s.hist[(b >> shift) & 255u], 1u);
+        uint32_t b;
+        if (key_of(j, b) && (b & mask) == prefix) atomicAdd(&s.hist[(b >> shift) & 255u], 1u);
       }
       __syncthreads();
       if (tid < 32) {  // lane l owns digits 8l .. 8l+7; find the digit holding the need-th largest
@@ -129,8 +126,94 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
       need = s.misc[1];
       __syncthreads();
     }
-    const uint32_t thr = prefix;
-    const int need_eq = need;
+    out_key = prefix;
+    out_need_eq = need;
+  };
+
+  if (target >= n_c) {
+    for (int r = tid; r < n_c; r += NT) s.src[r] = r;
+    __syncthreads();
+  } else if (e.recent) {  // Algorithm 3's rule: the most recent pairs stay, whatever their weights
+    for (int r = tid; r < target; r += NT) s.src[r] = n_c - target + r;
+    __syncthreads();
+  } else {
+    // ---- radix select: bit pattern `thr` of the target-th largest ave, and how many equal to it to keep
+    uint32_t thr;
+    int need_eq;
+    radix_kth_largest([&](int j, uint32_t& key) { key = ave_bits(j); return true; }, target, thr, need_eq);
+    if (c.fill) {
+      // ---- unordered cache: the rows of a cache are in no particular order, so (i) among the candidates equal to
+      // the cut the need_eq lowest positions stay, found by a second select on kv_ids, and (ii) nothing that stays
+      // moves: the candidates that stay but sit outside the first `target` rows (new pairs, and cached pairs beyond
+      // row `target`) fill the rows that are freed or empty, in ascending order on both sides.
+      const int eq_total = (int)s.hist[thr & 255u];   // the last pass counted the candidates equal to thr above the low digit
+      int id_cut = 0x7fffffff;
+      __syncthreads();   // the histogram is cleared by the next select
+      if (need_eq < eq_total) {
+        uint32_t key;
+        int unused;
+        radix_kth_largest([&](int j, uint32_t& k) { k = 0x7fffffffu - (uint32_t)s.id[j]; return ave_bits(j) == thr; },
+                          need_eq, key, unused);
+        id_cut = (int)(0x7fffffffu - key);
+      }
+      auto stays = [&](int j) { const uint32_t b = ave_bits(j); return b > thr || (b == thr && s.id[j] <= id_cut); };
+      const int chunk = (n_c + NT - 1) / NT;
+      const int jb = min(tid * chunk, n_c), je = min(jb + chunk, n_c);
+      int nfree = 0, nsrc = 0;
+      for (int j = jb; j < je; ++j) {
+        const bool k = stays(j);
+        nfree += (j < target && (j >= n_old || !k));
+        nsrc += (k && (j >= target || j >= n_old));
+      }
+      int fb, sb;
+      block_exclusive_scan2<NT>(nfree, nsrc, s.wsum, fb, sb);
+      int nf = 0;
+      for (int w = 0; w < NT / 32; ++w) nf += s.wsum[w];   // as many rows to fill as candidates to move
+      for (int j = jb; j < je; ++j) {
+        const bool k = stays(j);
+        if (j < target && (j >= n_old || !k)) s.dst[fb++] = j;
+        if (k && (j >= target || j >= n_old)) s.src[sb++] = j;
+      }
+      __syncthreads();
+      if (c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)nf);
+      for (int k = tid; k < nf; k += NT) {
+        const int j = s.src[k], r = s.dst[k];
+        c.sum_weights[base + r] = s.score[j];
+        c.kv_ids[base + r] = s.id[j];
+      }
+      // sources lie outside the first `target` rows, destinations inside: no row is both read and written
+      constexpr int PRF = D * (int)sizeof(T) / 16;
+      T* kslab = reinterpret_cast<T*>(c.k_slab) + base * D;
+      T* vslab = reinterpret_cast<T*>(c.v_slab) + base * D;
+      for (int x0 = 0; x0 < nf * PRF; x0 += 4 * NT) {
+        uint4 kb[4], vb[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const int x = x0 + t * NT + tid;
+          if (x < nf * PRF) {
+            const int j = s.src[x / PRF], pc = x % PRF;
+            if (j >= n_old) {
+              const size_t off = ((size_t)(smp * e.I + (j - n_old)) * c.Hkv + kh) * D;
+              kb[t] = ld_global_16(reinterpret_cast<const T*>(e.blk_k) + off + pc * (16 / sizeof(T)));
+              vb[t] = ld_global_16(reinterpret_cast<const T*>(e.blk_v) + off + pc * (16 / sizeof(T)));
+            } else {
+              kb[t] = ld_global_16(kslab + (size_t)j * D + pc * (16 / sizeof(T)));
+              vb[t] = ld_global_16(vslab + (size_t)j * D + pc * (16 / sizeof(T)));
+            }
+          }
+        }
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+          const int x = x0 + t * NT + tid;
+          if (x < nf * PRF) {
+            const int r = s.dst[x / PRF], pc = x % PRF;
+            st_global_16(kslab + (size_t)r * D + pc * (16 / sizeof(T)), kb[t]);
+            st_global_16(vslab + (size_t)r * D + pc * (16 / sizeof(T)), vb[t]);
+          }
+        }
+      }
+      return;
+    }
     // ---- stable destinations: candidates above thr, plus the first need_eq equal to thr (lower id first)
     const int chunk = (n_c + NT - 1) / NT;
     const int jb = min(tid * chunk, n_c), je = min(jb + chunk, n_c);

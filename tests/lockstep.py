@@ -23,8 +23,8 @@ OUT_TOL = {"bf16": 2e-2, "f32": 1e-4}
 
 
 def make_config(wl: Workload, device: int = 0, growth: int | None = None, batch: int | None = None,
-                max_call_samples: int = 0, rule: str = "average") -> Config:
-    return config_for(wl, device, growth, batch, max_call_samples, rule)
+                max_call_samples: int = 0, rule: str = "average", compaction: str = "stable") -> Config:
+    return config_for(wl, device, growth, batch, max_call_samples, rule, compaction)
 
 
 def _np(t):
@@ -69,12 +69,13 @@ def check_kept(unit: UnitCache, gpu_ids: np.ndarray, target: int, stats: dict, w
 
 
 def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=None, check_rows_every: int = 8,
-                 growth: int | None = None, sum_rtol: float | None = None, pads=None, rule: str = "average"):
+                 growth: int | None = None, sum_rtol: float | None = None, pads=None, rule: str = "average",
+                 compaction: str = "stable"):
     """Run `calls` (default: the workload's spec schedule) on the GPU for the whole batch and on the
     oracle for `units` = [(sample, kv_head), ...].  Returns a dict of statistics; raises on any mismatch."""
     dev = torch.device("cuda", device)
     inp = Inputs(wl, dev)
-    cfg = make_config(wl, device, growth, rule=rule)
+    cfg = make_config(wl, device, growth, rule=rule, compaction=compaction)
     cache = BatchMaxCache(cfg)
     if pads is not None:                            # left-padded samples: pads[sample] padding positions
         cache.set_left_pad(pads)
@@ -116,6 +117,12 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
             want_rows = (ci % check_rows_every == 0) or ci == len(calls) - 1
             ids, sw, kr, vr = cache.export(layer, smp, kh, rows=want_rows)
             ids = ids.numpy().astype(np.int64)
+            if compaction == "fill":                # an unordered cache exports its rows in storage order
+                order = np.argsort(ids, kind="stable")
+                assert len(np.unique(ids)) == len(ids), f"{where}: a position is cached twice"
+                ids, sw = ids[order], sw[torch.from_numpy(order)]
+                if want_rows:
+                    kr, vr = kr[torch.from_numpy(order)], vr[torch.from_numpy(order)]
             if kind != "recent" and evict_to >= 0 and len(unit) > evict_to:
                 check_kept(unit, ids, evict_to, stats, where)
             assert np.array_equal(ids, unit.kv_ids), f"{where}: kv_ids differ from the oracle's"

@@ -207,6 +207,102 @@ def test_decode_with_one_cache_per_sm(K, g):
     assert st["evictions"] >= 6 * 14
 
 
+# ------------------------------------------------------------------ unordered caches (BM_COMPACT_FILL)
+@pytest.mark.parametrize("name,kw", [
+    ("f32_simt", dict(dtype="f32", d=64, Hq=4, Hkv=4, s=300, B=48, K=80, steps=12)),
+    ("bf16_one_per_sm", dict(dtype="bf16", d=128, Hq=8, Hkv=2, s=700, B=128, K=512, steps=14)),
+    ("bf16_ragged_tail", dict(dtype="bf16", d=128, Hq=4, Hkv=4, s=333, B=100, K=77, steps=9)),
+    ("bf16_block_larger_than_cache", dict(dtype="bf16", d=64, Hq=2, Hkv=2, s=400, B=160, K=48, steps=6)),
+    ("bf16_decode_cuts_of_8", dict(dtype="bf16", d=128, Hq=8, Hkv=2, s=256, B=64, K=64, steps=20, p_dec=8)),
+])
+def test_unordered_cache_lockstep(name, kw):
+    # same kept sets, sums and outputs as the ordered cache; rows compared after sorting the export by position
+    wl = tiny("fill_" + name, **kw)
+    st = run_lockstep(wl, all_units(wl), compaction="fill", check_rows_every=1)
+    assert st["evictions"] > 0
+
+
+def test_unordered_cache_many_units_decode():
+    wl = tiny("fill_many", b=40, Hq=32, Hkv=8, s=160, B=64, K=72, steps=10, dtype="bf16", d=128)
+    run_lockstep(wl, [(0, 0), (13, 5), (39, 7), (27, 2)], compaction="fill", check_rows_every=2)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_unordered_cache_breaks_ties_by_position(dtype, d):
+    # A crafted state: rows in shuffled order, every sum_weights zero, one key (position 0) whose logit exceeds all
+    # others by more than 1000, so that every other weight underflows to exactly 0 in fp32 and in fp64 alike.  All
+    # those pairs tie at the cut; the lower positions must stay (select on kv_ids in the block eviction, arg-min on
+    # kv_ids in the decode step), pairs that stay must not move, and every row must keep its own position.
+    import torch
+    from paper_2412_05693_b200 import BatchMaxCache
+    from paper_2412_05693_b200.binding import Config
+    td = torch.bfloat16 if dtype == "bf16" else torch.float32
+    g, Hkv, K, n0 = 2, 2, 24, 32
+    cfg = Config(batch=1, n_q_heads=g * Hkv, n_kv_heads=Hkv, head_dim=d, kv_max=K, block_max=32, growth=40,
+                 dtype=dtype, compaction="fill")
+    cache = BatchMaxCache(cfg)
+    dev = torch.device("cuda", 0)
+    gen = torch.Generator().manual_seed(5)
+    rnd = lambda *shape: torch.randn(*shape, generator=gen).to(td).to(dev)
+    cache.prefill_block(rnd(1, n0, g * Hkv, d), rnd(1, n0, Hkv, d), rnd(1, n0, Hkv, d), 0, evict_to=-1)
+    perm = {}
+    for h in range(Hkv):
+        ids = torch.randperm(n0, generator=gen).to(torch.int32)
+        perm[h] = ids.tolist()
+        kr = torch.zeros(n0, d, dtype=td)
+        kr[ids == 0] = 10.0
+        vr = ids.to(td)[:, None].expand(n0, d).contiguous()      # a row's value is its position
+        cache.import_(ids, torch.zeros(n0), kr, vr, sample=0, kv_head=h)
+
+    def check(expect, before):
+        for h in range(Hkv):
+            ids, sw, kr, vr = cache.export(0, 0, h, rows=True)
+            ids = ids.tolist()
+            assert sorted(ids) == sorted(expect), f"head {h}: kept {sorted(ids)}, expected {sorted(expect)}"
+            assert torch.equal(vr[:, 0].float(), torch.tensor(ids, dtype=torch.float32)), "a row lost its position"
+            assert all(float(kr[r].float().abs().max()) == (10.0 if i in hot else 0.0) for r, i in enumerate(ids))
+            for r, i in enumerate(before[h][:len(ids)]):
+                if i in expect:
+                    assert ids[r] == i, f"head {h}: pair {i} stayed but moved from row {r}"
+            before[h] = ids
+
+    hot = {0}
+    q10 = lambda n: torch.full((1, n, g * Hkv, d), 10.0, dtype=td, device=dev)
+    vpos = lambda p0, n: torch.arange(p0, p0 + n, dtype=torch.float32)[None, :, None, None].expand(1, n, Hkv, d).to(td).to(dev)
+    # a block of 16: every pair but position 0 ties at zero -> positions 0..23 stay, the block's pairs all leave
+    cache.prefill_block(q10(16), torch.zeros(1, 16, Hkv, d, dtype=td, device=dev), vpos(n0, 16).contiguous(), n0, evict_to=K)
+    expect = list(range(K))
+    check(expect, perm)
+    # decode steps whose own key matches the query as well as position 0 does: the step's pair stays, and of the pairs
+    # tied at zero the highest position leaves
+    for t in range(6):
+        pos = n0 + 16 + t
+        cache.decode_step(q10(1)[:, 0].contiguous(), torch.full((1, Hkv, d), 10.0, dtype=td, device=dev),
+                          vpos(pos, 1)[:, 0].contiguous(), evict_to=K)
+        hot.add(pos)
+        expect.remove(max(i for i in expect if i not in hot))
+        expect.append(pos)
+        check(expect, perm)
+    assert cache.status() == 0
+    cache.close()
+
+
+def test_unordered_cache_rejects_what_needs_the_order():
+    import numpy as np
+    from paper_2412_05693_b200 import BatchMaxCache, BMError
+    from paper_2412_05693_b200.binding import Config
+    from tests.lockstep import make_config
+    wl = tiny("fill_rej", s=64, B=16, K=16, steps=1, dtype="bf16", d=128, Hq=4, Hkv=2)
+    with pytest.raises(BMError):
+        BatchMaxCache(make_config(wl, rule="sum_recent", compaction="fill"))
+    cache = BatchMaxCache(make_config(wl, compaction="fill"))
+    with pytest.raises(BMError):
+        cache.set_left_pad([0, 3])
+    with pytest.raises(BMError):
+        cache.keep_most_recent(1)
+    cache.close()
+
+
 # ------------------------------------------------------------------ the rules of Sec. 2 on the same kernels
 @pytest.mark.parametrize("rule", ["sum_recent", "current_query"])
 @pytest.mark.parametrize("dtype,d,Hq,Hkv", [("bf16", 128, 8, 2), ("f32", 64, 4, 4)])
