@@ -51,7 +51,7 @@ ARMS = {
 
 
 def make_cfg(wl: Workload, batch: int, arm: str, micro: int, device: int = 0, kv_bar: int | None = None,
-             p: int = 64) -> Config:
+             p: int = 64, compaction: str = "stable") -> Config:
     """Cache geometry of an arm; cap = kv_max + growth is what the memory model charges per cache."""
     block = wl.B
     if arm == "pd":
@@ -68,7 +68,8 @@ def make_cfg(wl: Workload, batch: int, arm: str, micro: int, device: int = 0, kv
         raise ValueError(arm)
     return Config(batch=batch, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.d, kv_max=kv_max, block_max=block,
                   growth=growth, dtype=wl.dtype, n_layers=wl.L, device=device,
-                  max_call_samples=max(micro, min(batch, DECODE_MICRO)))
+                  max_call_samples=max(micro, min(batch, DECODE_MICRO)),
+                  compaction="stable" if arm == "ed" else compaction)    # Algorithm 3's cut ranks rows by their order
 
 
 def arm_calls(wl: Workload, arm: str, kv_bar: int | None = None, p: int = 64):
@@ -172,10 +173,10 @@ class Timer:
 
 
 def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=None, device: int = 0,
-            kv_bar: int | None = None, p: int = 64):
+            kv_bar: int | None = None, p: int = 64, compaction: str = "stable"):
     """One arm (see ARMS) over the whole schedule.  Returns a dict of timings and derived rates."""
     wl = wl.with_(b=batch)
-    cfg = make_cfg(wl, batch, arm, micro, device, kv_bar, p)
+    cfg = make_cfg(wl, batch, arm, micro, device, kv_bar, p, compaction)
     dev = torch.device("cuda", device)
     need = arena_bytes(cfg)
     if arena is None:
@@ -259,7 +260,7 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
     dec_bytes = batch * wl.Hkv * n_layers * ((dec_rows / n_layers) * (2 * wl.d * e + 16)
                                              + wl.steps * (2 * wl.d * e + 2 * wl.g * wl.d * e))
     res = {
-        "workload": wl.name, "arm": arm, "batch": batch, "layers_run": n_layers, "micro_batch": micro,
+        "workload": wl.name, "arm": arm, "compaction": cfg.compaction, "batch": batch, "layers_run": n_layers, "micro_batch": micro,
         "decode_micro_batch": micro_dec, "cap": cfg.kv_max + cfg.growth,
         "arena_GiB": need / GiB, "final_n": n_end, "final_curr_id": cur,
         "prefill_ms": ms_pre, "decode_ms": ms_dec,
@@ -295,6 +296,8 @@ def main():
     ap.add_argument("--micro", type=int, default=256)
     ap.add_argument("--layers", type=int, default=None, help="run only the first N layers (cfg4)")
     ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--compaction", default="stable", choices=["stable", "fill"],
+                    help="fill: unordered caches (pairs that stay never move); Algorithm 3's arm always runs ordered")
     args = ap.parse_args()
     assert torch.cuda.is_available(), "needs a CUDA device (there is no CPU fallback)"
     torch.cuda.set_device(0)
@@ -306,11 +309,11 @@ def main():
         b_pd = max_batch(make_cfg(wl, 1, "pd", args.micro), budget)
         b_do = max_batch(make_cfg(wl, 1, "do", args.micro), budget)
         arena = torch.empty(budget, dtype=torch.uint8, device="cuda")
-        res_pd = run_arm(wl, b_pd, "pd", args.micro, arena=arena)
+        res_pd = run_arm(wl, b_pd, "pd", args.micro, arena=arena, compaction=args.compaction)
         out = {"run": args.run, "budget_GiB": budget / GiB, "b_pd": b_pd, "b_do": b_do,
                "batch_ratio": b_pd / b_do, "predicted_ratio": (wl.s + 1) / (wl.K + 1), "pd": res_pd}
         if args.run == "cfg3_ratio":
-            out["do"] = run_arm(wl, b_do, "do", min(args.micro, 64), arena=arena)
+            out["do"] = run_arm(wl, b_do, "do", min(args.micro, 64), arena=arena, compaction=args.compaction)
             out["generated_tok_s_ratio"] = out["pd"]["generated_tok_s"] / out["do"]["generated_tok_s"]
         print(json.dumps(out))
     elif args.run == "cfg4":
@@ -321,7 +324,7 @@ def main():
         b = max_batch(make_cfg(wl, 1, "pd", args.micro), budget)
         arena = torch.empty(budget, dtype=torch.uint8, device="cuda")
         layers = range(wl.L) if args.layers is None else range(args.layers)
-        res = run_arm(wl, b, "pd", args.micro, arena=arena, layers=layers)
+        res = run_arm(wl, b, "pd", args.micro, arena=arena, layers=layers, compaction=args.compaction)
         print(json.dumps({"run": "cfg4", "budget_GiB": budget / GiB, "batch": b, "pd": res}))
     elif args.run == "sec5":
         # The procedure of Sec. 5 on one attention layer of the larger model's shape (40 heads of 128, prompt
@@ -334,7 +337,7 @@ def main():
         arms = [("alg1", 1024), ("alg1", 2048), ("ed", 2), ("ed", 65), ("fkv", None)]
         for arm, kv_bar in arms:
             b = max_batch(make_cfg(wl, 1, arm, args.micro, kv_bar=kv_bar), budget)
-            res = run_arm(wl, b, arm, min(args.micro, b), arena=arena, kv_bar=kv_bar)
+            res = run_arm(wl, b, arm, min(args.micro, b), arena=arena, kv_bar=kv_bar, compaction=args.compaction)
             print(json.dumps({"run": "sec5", "budget_GiB": budget / GiB, "arm": arm, "kv_bar": kv_bar, "batch": b,
                               "result": res}), flush=True)
     else:
@@ -342,7 +345,7 @@ def main():
             wl = WORKLOADS["cfg5"].with_(B=B, K=K, name=f"cfg5_B{B}_K{K}")
             if args.decode_steps is not None:
                 wl = wl.with_(steps=args.decode_steps)
-            res = run_arm(wl, wl.b, "pd", wl.b)
+            res = run_arm(wl, wl.b, "pd", wl.b, compaction=args.compaction)
             print(json.dumps({"run": "cfg5", "block": B, "kv_max": K, "pd": res}), flush=True)
 
 
