@@ -67,7 +67,6 @@ bool config_ok(const bm_config_t* c, bool need_batch) {
   if (c->device < 0 || c->max_call_samples < 0) return false;
   if (c->rule < 0 || c->rule > 2) return false;
   if (c->compaction < 0 || c->compaction > 1) return false;
-  if (c->compaction == BM_COMPACT_FILL && c->rule != BM_RULE_AVERAGE) return false;
   if ((long long)c->kv_max + c->growth > (1 << 24)) return false;
   return true;
 }
@@ -407,7 +406,6 @@ bm_status_t bm_evict(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsam
 
 bm_status_t bm_keep_most_recent(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, int32_t keep,
                                 void* cuda_stream) {
-  if (c != nullptr && c->cfg.compaction == BM_COMPACT_FILL) return BM_ERR_INVALID;   // the rule ranks rows by their order
   return evict_cached(c, layer, sample0, nsamples, keep, true, cuda_stream);
 }
 

@@ -129,8 +129,10 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
   const size_t base = (size_t)unit * c.cap;
   T* kslab = reinterpret_cast<T*>(c.k_slab) + base * D;
   T* vslab = reinterpret_cast<T*>(c.v_slab) + base * D;
-  const bool evict_one = (a.target == n1 - 1);
-  const bool evict_general = (a.target >= 0 && a.target < n1 - 1);
+  // (an unordered cache under the rule with a window of recent pairs takes the general path for every cut: the
+  // window is a select on kv_ids there)
+  const bool evict_one = (a.target == n1 - 1) && (PLAIN || !(c.fill && c.rule == 1));
+  const bool evict_general = (a.target >= 0 && a.target < n1 && !evict_one);
 
   // Programmatic dependent launch: this grid may have been started while its predecessor in the stream was still
   // running (so that the launch latency of back-to-back decode steps is hidden); nothing that the predecessor may
@@ -705,7 +707,7 @@ cudaError_t launch_g(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
 
 size_t decode_mma_smem_bytes(int d, int g, int n_rows, int target) {
   const size_t attn = smem_layout(nullptr, d, g, n_rows, kMaxWarps, nullptr);
-  const size_t ev = (target >= 0 && target < n_rows - 1) ? evict_smem_bytes(n_rows, target) : 0;
+  const size_t ev = (target >= 0 && target < n_rows) ? evict_smem_bytes(n_rows, target) : 0;
   return attn > ev ? attn : ev;
 }
 

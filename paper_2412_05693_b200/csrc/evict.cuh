@@ -75,11 +75,12 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
   __syncthreads();
   const float gf = (float)c.g;
   const int pad = sample_left_pad(c, smp);
+  int id_win = 0x7fffffff;   // unordered cache, rule 1: pairs at positions >= id_win form the window of recent pairs
   auto ave_bits = [&](int j) -> uint32_t {
     const float cnt = (float)(e.curr_id + 1 - s.id[j]);
     uint32_t b;   // ranking value >= 0: the bit pattern orders like the value
     if (c.rule == 0) b = __float_as_uint(s.score[j] / (gf * cnt));       // average attention (Sec. 3.2)
-    else if (c.rule == 1 && j >= n_c - target / 2) b = 0x7f800000u;      // window of recent pairs: always kept
+    else if (c.rule == 1 && (c.fill ? s.id[j] >= id_win : j >= n_c - target / 2)) b = 0x7f800000u;   // recent window: always kept
     else b = __float_as_uint(s.score[j]);                                // raw (sum of / current) weights
     if (pad == 0) return b;
     return s.id[j] < pad ? 0u : max(b, 1u);   // padding pairs rank below every real pair (left-padded samples)
@@ -130,13 +131,87 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
     out_need_eq = need;
   };
 
+  // Unordered cache: nothing that stays moves.  The candidates that stay but sit outside the first `target` rows
+  // (new pairs, and cached pairs beyond row `target`) fill the rows that are freed or still empty, in ascending
+  // order on both sides.
+  auto fill_rows = [&](auto stays) {
+    const int chunk = (n_c + NT - 1) / NT;
+    const int jb = min(tid * chunk, n_c), je = min(jb + chunk, n_c);
+    int nfree = 0, nsrc = 0;
+    for (int j = jb; j < je; ++j) {
+      const bool k = stays(j);
+      nfree += (j < target && (j >= n_old || !k));
+      nsrc += (k && (j >= target || j >= n_old));
+    }
+    int fb, sb;
+    block_exclusive_scan2<NT>(nfree, nsrc, s.wsum, fb, sb);
+    int nf = 0;
+    for (int w = 0; w < NT / 32; ++w) nf += s.wsum[w];   // as many rows to fill as candidates to move
+    for (int j = jb; j < je; ++j) {
+      const bool k = stays(j);
+      if (j < target && (j >= n_old || !k)) s.dst[fb++] = j;
+      if (k && (j >= target || j >= n_old)) s.src[sb++] = j;
+    }
+    __syncthreads();
+    if (c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)nf);
+    for (int k = tid; k < nf; k += NT) {
+      const int j = s.src[k], r = s.dst[k];
+      c.sum_weights[base + r] = s.score[j];
+      c.kv_ids[base + r] = s.id[j];
+    }
+    // sources lie outside the first `target` rows, destinations inside: no row is both read and written
+    constexpr int PRF = D * (int)sizeof(T) / 16;
+    T* kslab = reinterpret_cast<T*>(c.k_slab) + base * D;
+    T* vslab = reinterpret_cast<T*>(c.v_slab) + base * D;
+    for (int x0 = 0; x0 < nf * PRF; x0 += 4 * NT) {
+      uint4 kb[4], vb[4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int x = x0 + t * NT + tid;
+        if (x < nf * PRF) {
+          const int j = s.src[x / PRF], pc = x % PRF;
+          if (j >= n_old) {
+            const size_t off = ((size_t)(smp * e.I + (j - n_old)) * c.Hkv + kh) * D;
+            kb[t] = ld_global_16(reinterpret_cast<const T*>(e.blk_k) + off + pc * (16 / sizeof(T)));
+            vb[t] = ld_global_16(reinterpret_cast<const T*>(e.blk_v) + off + pc * (16 / sizeof(T)));
+          } else {
+            kb[t] = ld_global_16(kslab + (size_t)j * D + pc * (16 / sizeof(T)));
+            vb[t] = ld_global_16(vslab + (size_t)j * D + pc * (16 / sizeof(T)));
+          }
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int x = x0 + t * NT + tid;
+        if (x < nf * PRF) {
+          const int r = s.dst[x / PRF], pc = x % PRF;
+          st_global_16(kslab + (size_t)r * D + pc * (16 / sizeof(T)), kb[t]);
+          st_global_16(vslab + (size_t)r * D + pc * (16 / sizeof(T)), vb[t]);
+        }
+      }
+    }
+  };
+
   if (target >= n_c) {
     for (int r = tid; r < n_c; r += NT) s.src[r] = r;
     __syncthreads();
+  } else if (e.recent && c.fill) {  // Algorithm 3's rule on an unordered cache: the `target` highest positions stay
+    uint32_t key = 0;
+    int unused;
+    if (target > 0) radix_kth_largest([&](int j, uint32_t& k) { k = (uint32_t)s.id[j]; return true; }, target, key, unused);
+    const int id_thr = target > 0 ? (int)key : 0x7fffffff;
+    fill_rows([&](int j) { return s.id[j] >= id_thr; });
+    return;
   } else if (e.recent) {  // Algorithm 3's rule: the most recent pairs stay, whatever their weights
     for (int r = tid; r < target; r += NT) s.src[r] = n_c - target + r;
     __syncthreads();
   } else {
+    if (c.fill && c.rule == 1 && target / 2 > 0) {   // the window's lowest position: the (target/2)-th highest
+      uint32_t key;
+      int unused;
+      radix_kth_largest([&](int j, uint32_t& k) { k = (uint32_t)s.id[j]; return true; }, target / 2, key, unused);
+      id_win = (int)key;
+    }
     // ---- radix select: bit pattern `thr` of the target-th largest ave, and how many equal to it to keep
     uint32_t thr;
     int need_eq;
@@ -156,62 +231,7 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
                           need_eq, key, unused);
         id_cut = (int)(0x7fffffffu - key);
       }
-      auto stays = [&](int j) { const uint32_t b = ave_bits(j); return b > thr || (b == thr && s.id[j] <= id_cut); };
-      const int chunk = (n_c + NT - 1) / NT;
-      const int jb = min(tid * chunk, n_c), je = min(jb + chunk, n_c);
-      int nfree = 0, nsrc = 0;
-      for (int j = jb; j < je; ++j) {
-        const bool k = stays(j);
-        nfree += (j < target && (j >= n_old || !k));
-        nsrc += (k && (j >= target || j >= n_old));
-      }
-      int fb, sb;
-      block_exclusive_scan2<NT>(nfree, nsrc, s.wsum, fb, sb);
-      int nf = 0;
-      for (int w = 0; w < NT / 32; ++w) nf += s.wsum[w];   // as many rows to fill as candidates to move
-      for (int j = jb; j < je; ++j) {
-        const bool k = stays(j);
-        if (j < target && (j >= n_old || !k)) s.dst[fb++] = j;
-        if (k && (j >= target || j >= n_old)) s.src[sb++] = j;
-      }
-      __syncthreads();
-      if (c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)nf);
-      for (int k = tid; k < nf; k += NT) {
-        const int j = s.src[k], r = s.dst[k];
-        c.sum_weights[base + r] = s.score[j];
-        c.kv_ids[base + r] = s.id[j];
-      }
-      // sources lie outside the first `target` rows, destinations inside: no row is both read and written
-      constexpr int PRF = D * (int)sizeof(T) / 16;
-      T* kslab = reinterpret_cast<T*>(c.k_slab) + base * D;
-      T* vslab = reinterpret_cast<T*>(c.v_slab) + base * D;
-      for (int x0 = 0; x0 < nf * PRF; x0 += 4 * NT) {
-        uint4 kb[4], vb[4];
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const int x = x0 + t * NT + tid;
-          if (x < nf * PRF) {
-            const int j = s.src[x / PRF], pc = x % PRF;
-            if (j >= n_old) {
-              const size_t off = ((size_t)(smp * e.I + (j - n_old)) * c.Hkv + kh) * D;
-              kb[t] = ld_global_16(reinterpret_cast<const T*>(e.blk_k) + off + pc * (16 / sizeof(T)));
-              vb[t] = ld_global_16(reinterpret_cast<const T*>(e.blk_v) + off + pc * (16 / sizeof(T)));
-            } else {
-              kb[t] = ld_global_16(kslab + (size_t)j * D + pc * (16 / sizeof(T)));
-              vb[t] = ld_global_16(vslab + (size_t)j * D + pc * (16 / sizeof(T)));
-            }
-          }
-        }
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-          const int x = x0 + t * NT + tid;
-          if (x < nf * PRF) {
-            const int r = s.dst[x / PRF], pc = x % PRF;
-            st_global_16(kslab + (size_t)r * D + pc * (16 / sizeof(T)), kb[t]);
-            st_global_16(vslab + (size_t)r * D + pc * (16 / sizeof(T)), vb[t]);
-          }
-        }
-      }
+      fill_rows([&](int j) { const uint32_t b = ave_bits(j); return b > thr || (b == thr && s.id[j] <= id_cut); });
       return;
     }
     // ---- stable destinations: candidates above thr, plus the first need_eq equal to thr (lower id first)

@@ -287,20 +287,52 @@ def test_unordered_cache_breaks_ties_by_position(dtype, d):
     cache.close()
 
 
-def test_unordered_cache_rejects_what_needs_the_order():
-    import numpy as np
+def test_unordered_cache_rejects_left_padding():
+    # cached padding is assumed to be a prefix of the rows (forward kernel's padding instance)
     from paper_2412_05693_b200 import BatchMaxCache, BMError
-    from paper_2412_05693_b200.binding import Config
     from tests.lockstep import make_config
     wl = tiny("fill_rej", s=64, B=16, K=16, steps=1, dtype="bf16", d=128, Hq=4, Hkv=2)
-    with pytest.raises(BMError):
-        BatchMaxCache(make_config(wl, rule="sum_recent", compaction="fill"))
     cache = BatchMaxCache(make_config(wl, compaction="fill"))
     with pytest.raises(BMError):
         cache.set_left_pad([0, 3])
-    with pytest.raises(BMError):
-        cache.keep_most_recent(1)
+    cache.set_left_pad([0, 0])
     cache.close()
+
+
+@pytest.mark.parametrize("rule", ["sum_recent", "current_query"])
+@pytest.mark.parametrize("dtype,d,Hq,Hkv,p_dec", [("bf16", 128, 8, 2, 1), ("f32", 64, 4, 4, 1), ("bf16", 128, 8, 2, 8)])
+def test_unordered_cache_alternative_rules(rule, dtype, d, Hq, Hkv, p_dec):
+    # the window of recent pairs is a select on kv_ids here, in the block eviction and in the decode step alike
+    wl = tiny("fill_rules", s=400, B=128, K=96, steps=12, dtype=dtype, d=d, Hq=Hq, Hkv=Hkv, p_dec=p_dec)
+    run_lockstep(wl, all_units(wl), rule=rule, compaction="fill", check_rows_every=2)
+
+
+@pytest.mark.parametrize("kv_bar", [2, 33])
+def test_unordered_cache_extreme_decoding_arm(kv_bar):
+    # Algorithm 3's cut keeps the highest positions, wherever their rows are
+    s, gen = 200, 70
+    wl = tiny("fill_ed", s=s, B=48, K=s, steps=gen, dtype="bf16", d=128, Hq=8, Hkv=2)
+    calls = [("prefill", t, min(48, s - t), -1) for t in range(0, s, 48)] + [("recent", 0, 0, 1)]
+    n = 1
+    for t in range(gen):
+        calls.append(("decode", s + t, 1, -1))
+        n += 1
+        if n == kv_bar:
+            calls.append(("recent", 0, 0, 1))
+            n = 1
+    run_lockstep(wl, all_units(wl), calls=calls, growth=kv_bar, compaction="fill", check_rows_every=5)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_unordered_cache_random_cadences(seed):
+    rng = np.random.default_rng(9100 + seed)
+    g, hkv, d = int(rng.choice([1, 2, 4, 8])), int(rng.integers(1, 4)), int(rng.choice([64, 128]))
+    wl = Workload(f"fillcad{seed}", b=int(rng.integers(1, 4)), Hq=g * hkv, Hkv=hkv, d=d, dtype=str(rng.choice(["bf16", "f32"])),
+                  s=int(rng.integers(50, 900)), B=int(rng.integers(1, 300)), K=int(rng.integers(1, 400)),
+                  steps=int(rng.integers(0, 16)), seed=9100 + seed, heavy_count=3, p_dec=int(rng.choice([1, 3])))
+    rule = str(rng.choice(["average", "sum_recent", "current_query"]))
+    calls, growth = random_cadence(wl, rng)     # prefill / decode / evict / recency cuts in any order
+    run_lockstep(wl, all_units(wl)[:3], calls=calls, growth=growth, rule=rule, compaction="fill", check_rows_every=3)
 
 
 # ------------------------------------------------------------------ the rules of Sec. 2 on the same kernels
