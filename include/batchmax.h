@@ -71,8 +71,7 @@ typedef enum { BM_RULE_AVERAGE = 0, BM_RULE_SUM_RECENT = 1, BM_RULE_CURRENT_QUER
  *                      kept pairs, the decode step's pair) take the rows that were freed.  Kept sets, sum_weights and
  *                      outputs are the same as under BM_COMPACT_STABLE (ties still keep the lower position, decided
  *                      on kv_ids; the recent window of BM_RULE_SUM_RECENT and bm_keep_most_recent rank by kv_ids);
- *                      bm_cache_export returns the rows in storage order.  bm_cache_set_left_pad with a non-zero
- *                      count returns BM_ERR_INVALID (cached padding is assumed to be a prefix of the rows). */
+ *                      bm_cache_export returns the rows in storage order. */
 typedef enum { BM_COMPACT_STABLE = 0, BM_COMPACT_FILL = 1 } bm_compaction_t;
 
 /* Problem statement: Algorithm 1's inputs (\overline{|kv|}, p) generalised as (K, growth), plus the

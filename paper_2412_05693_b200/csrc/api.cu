@@ -549,7 +549,6 @@ bm_status_t bm_cache_set_left_pad(bm_cache_t* c, const int32_t* pads, void* cuda
       if (pads[s] < 0) return BM_ERR_INVALID;
       any = any || pads[s] > 0;
     }
-  if (any && c->cfg.compaction == BM_COMPACT_FILL) return BM_ERR_INVALID;   // padding is a prefix of an ordered cache
   c->has_pad = any;
   if (!any) return BM_OK;
   c->pad_host.assign(pads, pads + c->cfg.batch);

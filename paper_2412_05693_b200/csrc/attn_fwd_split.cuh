@@ -32,7 +32,8 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + L::kBars);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* np_slot = reinterpret_cast<int*>(tmem_slot + 2);   // cached padding pairs of the unit
+  // [2][4] words: which keys of a cached tile are padding pairs (double-buffered over key tiles)
+  uint32_t* pmask = reinterpret_cast<uint32_t*>(sm + L::kBars + 128);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int unit = blockIdx.y, smp = unit / a.Hkv, kh = unit % a.Hkv;
@@ -60,7 +61,6 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
   };
   if (warp == kTmaWarp && lane == 0) {
     *abort_flag = 0;
-    *np_slot = 0;
     mbar_init(&bars[B_QFULL], 1);
     mbar_init(&bars[B_SFULL], 1);
     mbar_init(&bars[B_PFULL], 256);
@@ -140,18 +140,23 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
     const int row = row0 + r;
     const int i_row = min(a.I - 1, i0 + r / a.g);  // rows past the block's end behave like its last input
     const int c_lo = 64 * half;                   // first key column of this thread
-    int pad = 0, n_pad = 0;
-    if (PAD) {                                    // cached padding pairs = the first n_pad rows (ids ascend)
+    // Left padding: a padding pair is masked for every real query.  Among the block's own keys padding is a prefix
+    // of positions; among the cached pairs it is whatever kv_ids say (the rows of an unordered cache are in no
+    // order), so warps 0-3 turn the kv_ids of each cached tile into a 128-bit mask one tile ahead.
+    int pad = 0;
+    const int* ids = a.kv_ids + (size_t)unit * a.cap;
+    auto publish_pad_mask = [&](int jt) {   // tile jt < t_old, by the 128 threads of half 0
+      if (half == 0) {
+        const int k = jt * kTileN + r;
+        const uint32_t w = __ballot_sync(0xffffffffu, k < a.n_old && ids[k] < pad);
+        if (lane == 0) pmask[(jt & 1) * 4 + quad] = w;
+      }
+    };
+    if (PAD) {
       pad = a.left_pad[smp];
-      const int* ids = a.kv_ids + (size_t)unit * a.cap;
-      if (pad > 0 && a.n_old > 0 && ids[0] < pad) {
-        int cnt = 0;
-        for (int t = tid; t < min(a.n_old, pad); t += 256) cnt += ids[t] < pad;
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
-        if (lane == 0 && cnt > 0) atomicAdd(np_slot, cnt);
+      if (pad > 0 && t_old > 0) {
+        publish_pad_mask(0);
         named_bar_sync(1, 256);
-        n_pad = *np_slot;
       }
     }
     const bool real_row = !PAD || a.pos0 + i_row >= pad;
@@ -162,10 +167,14 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
       // visible columns of this key tile for this row: [nlo, nvis)
       const int nvis = (j < t_old) ? min(kTileN, a.n_old - j * kTileN)
                                    : max(0, min(kTileN, i_row - (j - t_old) * kTileN + 1));
-      const int nlo = (!PAD || !real_row) ? 0
-                      : (j < t_old) ? max(0, min(kTileN, n_pad - j * kTileN))
-                                    : max(0, min(kTileN, pad - a.pos0 - (j - t_old) * kTileN));
-      const bool full = __all_sync(0xffffffffu, nvis >= kTileN && nlo == 0);   // warp-uniform: nothing to mask
+      // padding among this thread's 64 columns: a prefix [0, nlo) of a block tile, a bit mask of a cached tile
+      const int nlo = (!PAD || !real_row || j < t_old) ? 0 : max(0, min(kTileN, pad - a.pos0 - (j - t_old) * kTileN));
+      uint64_t pm = 0;
+      if (PAD && pad > 0 && j < t_old) {
+        if (real_row) pm = (uint64_t)pmask[(j & 1) * 4 + 2 * half] | ((uint64_t)pmask[(j & 1) * 4 + 2 * half + 1] << 32);
+        if (j + 1 < t_old) publish_pad_mask(j + 1);   // read after this tile's exchange of maxima (a barrier)
+      }
+      const bool full = __all_sync(0xffffffffu, nvis >= kTileN && nlo == 0 && pm == 0);   // warp-uniform: nothing to mask
       uint32_t s0[32], s1[32];
       tmem_ld32(tm_s + lane_addr + c_lo, s0);
       tmem_ld32(tm_s + lane_addr + c_lo + 32, s1);
@@ -181,8 +190,8 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
           const int c0 = c_lo + e, c1 = c_lo + 32 + e;
-          mx = fmaxf(mx, (c0 < nvis && c0 >= nlo) ? __uint_as_float(s0[e]) : -INFINITY);
-          mx = fmaxf(mx, (c1 < nvis && c1 >= nlo) ? __uint_as_float(s1[e]) : -INFINITY);
+          mx = fmaxf(mx, (c0 < nvis && c0 >= nlo && !((pm >> e) & 1)) ? __uint_as_float(s0[e]) : -INFINITY);
+          mx = fmaxf(mx, (c1 < nvis && c1 >= nlo && !((pm >> (32 + e)) & 1)) ? __uint_as_float(s1[e]) : -INFINITY);
         }
       }
       // the row's other thread holds the maximum of the other 64 columns
@@ -224,8 +233,8 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
           float p0 = ex2(x0), p1 = ex2(x1);
           if (!full) {
             const int c0 = c_lo + 32 * ch + 2 * e;
-            p0 = (c0 < nvis && c0 >= nlo) ? p0 : 0.f;
-            p1 = (c0 + 1 < nvis && c0 + 1 >= nlo) ? p1 : 0.f;
+            p0 = (c0 < nvis && c0 >= nlo && !((pm >> (32 * ch + 2 * e)) & 1)) ? p0 : 0.f;
+            p1 = (c0 + 1 < nvis && c0 + 1 >= nlo && !((pm >> (32 * ch + 2 * e + 1)) & 1)) ? p1 : 0.f;
           }
           add2(ps0, ps1, p0, p1);
           pk[e] = pack_bf16(p0, p1);

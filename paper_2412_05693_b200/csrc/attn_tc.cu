@@ -646,7 +646,8 @@ int g_fwd_kernel = 0;   // 0: two threads per row; 1 / 2: one thread per row, on
 
 template <int D>
 cudaError_t launch_fwd_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
-  if (g_fwd_kernel == 0)
+  // (the one-thread-per-row kernels take cached padding to be a prefix of the rows: not so in an unordered cache)
+  if (g_fwd_kernel == 0 || (c.fill && c.left_pad != nullptr))
     return c.left_pad != nullptr ? launch_fwd_split<D, true>(c, a, st) : launch_fwd_split<D, false>(c, a, st);
   if (c.left_pad != nullptr)
     return g_fwd_tiles_override == 2 ? launch_fwd_nt<D, 2, true>(c, a, st) : launch_fwd_nt<D, 1, true>(c, a, st);

@@ -287,16 +287,17 @@ def test_unordered_cache_breaks_ties_by_position(dtype, d):
     cache.close()
 
 
-def test_unordered_cache_rejects_left_padding():
-    # cached padding is assumed to be a prefix of the rows (forward kernel's padding instance)
-    from paper_2412_05693_b200 import BatchMaxCache, BMError
-    from tests.lockstep import make_config
-    wl = tiny("fill_rej", s=64, B=16, K=16, steps=1, dtype="bf16", d=128, Hq=4, Hkv=2)
-    cache = BatchMaxCache(make_config(wl, compaction="fill"))
-    with pytest.raises(BMError):
-        cache.set_left_pad([0, 3])
-    cache.set_left_pad([0, 0])
-    cache.close()
+@pytest.mark.parametrize("dtype,d,s,B,K,pads", [
+    ("f32", 64, 200, 48, 40, [0, 37, 150]),
+    ("bf16", 128, 600, 128, 160, [0, 301, 77]),     # cached padding scattered over the rows of several key tiles
+    ("bf16", 128, 333, 100, 77, [5, 250, 0]),
+    ("bf16", 64, 256, 64, 300, [0, 200, 64]),       # nothing leaves during the prompt: padding stays cached in decoding
+])
+def test_unordered_cache_left_padding(dtype, d, s, B, K, pads):
+    # padding pairs are masked by their kv_ids wherever their rows are, and leave first
+    wl = tiny("fill_pad", b=3, s=s, B=B, K=K, steps=8, dtype=dtype, d=d, Hq=8 if d == 128 else 4, Hkv=2)
+    run_lockstep(wl, all_units(wl), pads=pads, compaction="fill", check_rows_every=2)
+    run_lockstep(wl, all_units(wl), pads=pads, compaction="fill", rule="sum_recent", check_rows_every=4)
 
 
 @pytest.mark.parametrize("rule", ["sum_recent", "current_query"])
@@ -331,8 +332,12 @@ def test_unordered_cache_random_cadences(seed):
                   s=int(rng.integers(50, 900)), B=int(rng.integers(1, 300)), K=int(rng.integers(1, 400)),
                   steps=int(rng.integers(0, 16)), seed=9100 + seed, heavy_count=3, p_dec=int(rng.choice([1, 3])))
     rule = str(rng.choice(["average", "sum_recent", "current_query"]))
-    calls, growth = random_cadence(wl, rng)     # prefill / decode / evict / recency cuts in any order
-    run_lockstep(wl, all_units(wl)[:3], calls=calls, growth=growth, rule=rule, compaction="fill", check_rows_every=3)
+    if seed % 2 == 0:
+        calls, growth = random_cadence(wl, rng)     # prefill / decode / evict / recency cuts in any order
+        run_lockstep(wl, all_units(wl)[:3], calls=calls, growth=growth, rule=rule, compaction="fill", check_rows_every=3)
+    else:
+        pads = [int(rng.integers(0, wl.s + 1)) for _ in range(wl.b)]
+        run_lockstep(wl, all_units(wl)[:3], pads=pads, rule=rule, compaction="fill", check_rows_every=3)
 
 
 # ------------------------------------------------------------------ the rules of Sec. 2 on the same kernels
