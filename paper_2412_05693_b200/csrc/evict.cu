@@ -7,22 +7,27 @@ namespace {
 
 constexpr int kEvictThreads = 512;
 
-template <typename T, int D>
+template <typename T, int D, bool FILL>
 __global__ void __launch_bounds__(kEvictThreads) evict_kernel(CacheView c, EvictArgs e) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int unit = blockIdx.x;
-  evict_body<T, D, kEvictThreads>(c, unit, unit / c.Hkv, unit % c.Hkv, e, smem_raw);
+  evict_body_impl<T, D, kEvictThreads, FILL>(c, unit, unit / c.Hkv, unit % c.Hkv, e, smem_raw);
+}
+
+template <typename T, int D, bool FILL>
+cudaError_t launch_f(const CacheView& c, const EvictArgs& e, cudaStream_t st) {
+  const size_t smem = evict_smem_bytes(c.n_old + e.I, e.target);
+  static SmemConfigured configured;
+  if (cudaError_t err = configured.ensure(evict_kernel<T, D, FILL>, smem); err != cudaSuccess) return err;
+  ProfileScope prof(kEvict, st);
+  evict_kernel<T, D, FILL><<<c.nsamples * c.Hkv, kEvictThreads, smem, st>>>(c, e);
+  count_launch();
+  return cudaGetLastError();
 }
 
 template <typename T, int D>
 cudaError_t launch_t(const CacheView& c, const EvictArgs& e, cudaStream_t st) {
-  const size_t smem = evict_smem_bytes(c.n_old + e.I, e.target);
-  static SmemConfigured configured;
-  if (cudaError_t err = configured.ensure(evict_kernel<T, D>, smem); err != cudaSuccess) return err;
-  ProfileScope prof(kEvict, st);
-  evict_kernel<T, D><<<c.nsamples * c.Hkv, kEvictThreads, smem, st>>>(c, e);
-  count_launch();
-  return cudaGetLastError();
+  return c.fill ? launch_f<T, D, true>(c, e, st) : launch_f<T, D, false>(c, e, st);
 }
 
 }  // namespace

@@ -13,6 +13,7 @@ namespace bm {
 
 struct EvictSmem {
   float* score;    // [n_cand]
+  uint32_t* bits;  // [n_cand]   ranking value of every candidate as an ordered bit pattern (computed once)
   int32_t* id;     // [n_cand]
   int32_t* src;    // [target]   candidate index that lands in row r (fill mode: k-th candidate that has to move)
   int32_t* dst;    // [target]   fill mode: row the k-th moving candidate lands in
@@ -25,11 +26,13 @@ __host__ __device__ inline size_t evict_smem_layout(unsigned char* base, int n_c
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) & ~size_t(15); return o; };
   size_t o_score = take(sizeof(float) * n_cand), o_id = take(sizeof(int32_t) * n_cand);
+  size_t o_bits = take(sizeof(uint32_t) * n_cand);
   size_t o_src = take(sizeof(int32_t) * (target > 0 ? target : 1)), o_dst = take(sizeof(int32_t) * (target > 0 ? target : 1));
   size_t o_hist = take(sizeof(uint32_t) * 256);
   size_t o_misc = take(sizeof(int32_t) * 8), o_wsum = take(sizeof(int32_t) * 64);
   if (s != nullptr) {
     s->score = reinterpret_cast<float*>(base + o_score);
+    s->bits = reinterpret_cast<uint32_t*>(base + o_bits);
     s->id = reinterpret_cast<int32_t*>(base + o_id);
     s->src = reinterpret_cast<int32_t*>(base + o_src);
     s->dst = reinterpret_cast<int32_t*>(base + o_dst);
@@ -59,8 +62,10 @@ __device__ inline void block_exclusive_scan2(int a, int b, int32_t* wsum /*[64]*
   __syncthreads();
 }
 
-template <typename T, int D, int NT>
-__device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh, const EvictArgs& e,
+// FILL: the cache's rows are an unordered set (CacheView::fill); a template parameter, so that the instance for
+// ordered rows carries none of that code (with both in one function the ordered instance ran 15 % slower).
+template <typename T, int D, int NT, bool FILL>
+__device__ inline void evict_body_impl(const CacheView& c, int unit, int smp, int kh, const EvictArgs& e,
                                   unsigned char* smem_raw) {
   const int tid = threadIdx.x;
   const int n_old = c.n_old, n_c = c.n_old + e.I, target = e.target;
@@ -80,7 +85,7 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
     const float cnt = (float)(e.curr_id + 1 - s.id[j]);
     uint32_t b;   // ranking value >= 0: the bit pattern orders like the value
     if (c.rule == 0) b = __float_as_uint(s.score[j] / (gf * cnt));       // average attention (Sec. 3.2)
-    else if (c.rule == 1 && (c.fill ? s.id[j] >= id_win : j >= n_c - target / 2)) b = 0x7f800000u;   // recent window: always kept
+    else if (c.rule == 1 && (FILL ? s.id[j] >= id_win : j >= n_c - target / 2)) b = 0x7f800000u;   // recent window: always kept
     else b = __float_as_uint(s.score[j]);                                // raw (sum of / current) weights
     if (pad == 0) return b;
     return s.id[j] < pad ? 0u : max(b, 1u);   // padding pairs rank below every real pair (left-padded samples)
@@ -195,7 +200,7 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
   if (target >= n_c) {
     for (int r = tid; r < n_c; r += NT) s.src[r] = r;
     __syncthreads();
-  } else if (e.recent && c.fill) {  // Algorithm 3's rule on an unordered cache: the `target` highest positions stay
+  } else if (FILL && e.recent) {  // Algorithm 3's rule on an unordered cache: the `target` highest positions stay
     uint32_t key = 0;
     int unused;
     if (target > 0) radix_kth_largest([&](int j, uint32_t& k) { k = (uint32_t)s.id[j]; return true; }, target, key, unused);
@@ -206,7 +211,7 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
     for (int r = tid; r < target; r += NT) s.src[r] = n_c - target + r;
     __syncthreads();
   } else {
-    if (c.fill && c.rule == 1 && target / 2 > 0) {   // the window's lowest position: the (target/2)-th highest
+    if (FILL && c.rule == 1 && target / 2 > 0) {   // the window's lowest position: the (target/2)-th highest
       uint32_t key;
       int unused;
       radix_kth_largest([&](int j, uint32_t& k) { k = (uint32_t)s.id[j]; return true; }, target / 2, key, unused);
@@ -215,8 +220,10 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
     // ---- radix select: bit pattern `thr` of the target-th largest ave, and how many equal to it to keep
     uint32_t thr;
     int need_eq;
-    radix_kth_largest([&](int j, uint32_t& key) { key = ave_bits(j); return true; }, target, thr, need_eq);
-    if (c.fill) {
+    for (int j = tid; j < n_c; j += NT) s.bits[j] = ave_bits(j);   // one division per candidate, not one per pass
+    __syncthreads();
+    radix_kth_largest([&](int j, uint32_t& key) { key = s.bits[j]; return true; }, target, thr, need_eq);
+    if constexpr (FILL) {
       // ---- unordered cache: the rows of a cache are in no particular order, so (i) among the candidates equal to
       // the cut the need_eq lowest positions stay, found by a second select on kv_ids, and (ii) nothing that stays
       // moves: the candidates that stay but sit outside the first `target` rows (new pairs, and cached pairs beyond
@@ -227,11 +234,11 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
       if (need_eq < eq_total) {
         uint32_t key;
         int unused;
-        radix_kth_largest([&](int j, uint32_t& k) { k = 0x7fffffffu - (uint32_t)s.id[j]; return ave_bits(j) == thr; },
+        radix_kth_largest([&](int j, uint32_t& k) { k = 0x7fffffffu - (uint32_t)s.id[j]; return s.bits[j] == thr; },
                           need_eq, key, unused);
         id_cut = (int)(0x7fffffffu - key);
       }
-      fill_rows([&](int j) { const uint32_t b = ave_bits(j); return b > thr || (b == thr && s.id[j] <= id_cut); });
+      fill_rows([&](int j) { const uint32_t b = s.bits[j]; return b > thr || (b == thr && s.id[j] <= id_cut); });
       return;
     }
     // ---- stable destinations: candidates above thr, plus the first need_eq equal to thr (lower id first)
@@ -239,14 +246,14 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
     const int jb = min(tid * chunk, n_c), je = min(jb + chunk, n_c);
     int gt = 0, eq = 0;
     for (int j = jb; j < je; ++j) {
-      const uint32_t b = ave_bits(j);
+      const uint32_t b = s.bits[j];
       gt += (b > thr);
       eq += (b == thr);
     }
     int gt_before, eq_before;
     block_exclusive_scan2<NT>(gt, eq, s.wsum, gt_before, eq_before);
     for (int j = jb; j < je; ++j) {
-      const uint32_t b = ave_bits(j);
+      const uint32_t b = s.bits[j];
       if (b > thr) { s.src[gt_before + min(eq_before, need_eq)] = j; ++gt_before; }
       else if (b == thr) {
         if (eq_before < need_eq) s.src[gt_before + eq_before] = j;
@@ -314,6 +321,13 @@ __device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh,
       }
     }
   }
+}
+
+template <typename T, int D, int NT>
+__device__ inline void evict_body(const CacheView& c, int unit, int smp, int kh, const EvictArgs& e,
+                                  unsigned char* smem_raw) {
+  if (c.fill) evict_body_impl<T, D, NT, true>(c, unit, smp, kh, e, smem_raw);
+  else evict_body_impl<T, D, NT, false>(c, unit, smp, kh, e, smem_raw);
 }
 
 }  // namespace bm
