@@ -640,11 +640,12 @@ template <int D, int G, int NT>
 cudaError_t launch_nt(const CacheView& c, const DecodeArgs& a, cudaStream_t st, bool one_per_sm) {
   const bool plain = c.left_pad == nullptr && c.rule == 0;
   if constexpr (NT == 256 && D == 128) {
-    if (plain && one_per_sm && c.n_old + 1 <= kBatchTiles * (NT / 32) * 16 &&
+    if (one_per_sm && c.n_old + 1 <= kBatchTiles * (NT / 32) * 16 &&
         decode_mma_smem_bytes(D, G, c.n_old + 1, a.target) + stage_bytes(D, NT, kBatchTiles) <= kMaxDynamicSmem) {
       CUtensorMap vmap;
       if (encode_slab_rows_map(&vmap, c.v_slab, D, c.n_old, c.cap, c.nsamples * c.Hkv, 128))
-        return launch_nt_p<D, G, NT, true, kBatchTiles>(c, a, st, vmap);
+        return plain ? launch_nt_p<D, G, NT, true, kBatchTiles>(c, a, st, vmap)
+                     : launch_nt_p<D, G, NT, false, kBatchTiles>(c, a, st, vmap);
     }
   }
   static const CUtensorMap no_map = {};   // the other instances take no tensor map
