@@ -31,15 +31,17 @@ def test_cfg1_everything():
     assert st["max_out_err"] <= 1e-4
 
 
-def test_cfg2_full_size_sampled_units():
+@pytest.mark.parametrize("compaction", ["stable", "fill"])
+def test_cfg2_full_size_sampled_units(compaction):
     wl = WORKLOADS["cfg2"]
-    st = run_lockstep(wl, [(0, 0), (7, 3), (15, 7)], check_rows_every=16)
+    st = run_lockstep(wl, [(0, 0), (7, 3), (15, 7)], check_rows_every=16, compaction=compaction)
     assert st["evictions"] > 0 and st["max_out_err"] <= 2e-2
 
 
-def test_cfg3_full_size_sampled_units():
+@pytest.mark.parametrize("compaction", ["stable", "fill"])
+def test_cfg3_full_size_sampled_units(compaction):
     wl = WORKLOADS["cfg3"].with_(steps=8)
-    run_lockstep(wl, [(3, 1), (12, 6)], check_rows_every=8)
+    run_lockstep(wl, [(3, 1), (12, 6)], check_rows_every=8, compaction=compaction)
 
 
 def test_cfg3_decode_only_compression_arm():
@@ -60,6 +62,7 @@ def test_cfg4_layers_are_independent():
 def test_cfg5_large_candidate_sets(B, K):
     wl = WORKLOADS["cfg5"].with_(b=2, B=B, K=K, s=8192, steps=4)
     run_lockstep(wl, [(1, 17)], check_rows_every=4)
+    run_lockstep(wl, [(0, 30)], check_rows_every=4, compaction="fill")
 
 
 def test_cfg5_full_length_prompt():
