@@ -7,6 +7,9 @@
 // Both contractions are invariant under a permutation of the contracted index, and the output index of the
 // second one can be un-permuted when it is written, so every thread loads whole 16-byte pieces of cache
 // rows (coalesced) and the MMA fragment slots are assigned to whatever elements those loads delivered.
+// The instance for grids of at most one cache per SM (KD > 1 below) differs in how rows travel: K is loaded once and
+// kept in registers, V is staged in shared memory by TMA while the softmax phases run and read back with
+// transposing ldmatrix (standard fragment layout), and the rows behind the pair that leaves are written from there.
 #include <cstdlib>
 
 #include "evict.cuh"
