@@ -50,6 +50,10 @@ def parse_args():
     ap.add_argument("--compaction", default="stable", choices=["stable", "fill"],
                     help="stable: a cache's rows stay in position order (rows behind a pair that leaves move up); "
                          "fill: unordered rows, pairs that stay never move (same kept sets and outputs)")
+    ap.add_argument("--ranges", type=int, default=4,
+                    help="split the batch into this many sample ranges, each range's calls on a stream of its own (all "
+                         "inside the step's graph): the caches of different samples are independent, so the tail of one "
+                         "range's kernel overlaps the next kernel of another range")
     ap.add_argument("--ragged", action="store_true",
                     help="left-padded samples: seeded padding counts in [0, s/2] (sample 0 unpadded); launches eagerly")
     return ap.parse_args()
@@ -259,10 +263,39 @@ def main():
         pads = [0] + [rng.randrange(0, wl.s // 2 + 1) for _ in range(wl.b - 1)]
         args.no_graph = True     # the padding counts are copied from pageable host memory at the start of a step
 
-    def one_step(host_bufs=None, with_decode=True, moved=None):
+    n_ranges = args.ranges if (args.ranges > 1 and wl.b % args.ranges == 0 and pads is None) else 1
+    side = [torch.cuda.Stream(device=dev) for _ in range(n_ranges)] if n_ranges > 1 else []
+
+    def step_in_ranges(cache, with_decode):
+        """The same calls, one sample range per stream; forked from and joined to the current stream."""
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        nb = wl.b // n_ranges
+        for r, st in enumerate(side):
+            st.wait_event(fork)
+            sl = slice(r * nb, (r + 1) * nb)
+            with torch.cuda.stream(st):
+                for layer in range(wl.L):
+                    for ci, (kind, pos0, I, ev) in enumerate(calls):
+                        q, k, v = dev_in[ci]
+                        if kind == "prefill":
+                            cache.prefill_block(q[sl], k[sl], v[sl], pos0, out=out_blk[sl, :I], evict_to=ev, layer=layer,
+                                                sample0=r * nb)
+                        elif with_decode:
+                            cache.decode_step(q[sl], k[sl], v[sl], out=out_dec[sl], evict_to=ev, layer=layer,
+                                              sample0=r * nb)
+            join = torch.cuda.Event()
+            join.record(st)
+            main.wait_event(join)
+
+    def one_step(host_bufs=None, with_decode=True, moved=None, ranges=True):
         cache = bm.BatchMaxCache(cfg_now[0], arena=arena, workspace=workspace)
         if pads is not None:
             cache.set_left_pad(pads)
+        if n_ranges > 1 and ranges and host_bufs is None and moved is None:
+            step_in_ranges(cache, with_decode)
+            return cache
         if moved is not None:                 # count the rows the compactions move, prefill and decode apart
             cache.count_moved_rows(True)
         for layer in range(wl.L):
@@ -345,7 +378,7 @@ def main():
     value = whole_job_value(tokens, world, ms_step)
 
     # ---- rooflines: every launch of an extra eager pass is bracketed by CUDA events inside the library
-    prof = bm.binding.profile_pass(lambda: one_step().close())
+    prof = bm.binding.profile_pass(lambda: one_step(ranges=False).close())   # whole-batch calls, one after the other
     pk, pk_src = peaks()
     extra = {"kernel_ms_per_step": {k: v[0] for k, v in prof.items()},
              "kernel_launches_per_step": {k: v[1] for k, v in prof.items()}}
@@ -384,6 +417,9 @@ def main():
             "achieved_with_compaction_writes": (dec_bytes + move_bytes) / (in_region_ms * 1e-3) / 1e9,
             "rows_moved_per_cache_and_step": moved.get("decode", 0) / max(1, wl.b * wl.Hkv * dec_n),
             "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(wl.name, {}).get("decode"),
+            "in_timed_region": (f"every decode step runs as {n_ranges} concurrent launches, one per sample range; "
+                                "achieved = bytes of all of them / their time in the region") if n_ranges > 1 else
+                               "one launch per decode step",
             "peak_source": f"{pk_src} (HBM copy)", "launches_per_step": dec_n,
             "avg_launch_ms": dec_ms / max(dec_n, 1),
             "algorithmic": "(n+1)*(2*d*e+16) + 2*d*e + 2*g*d*e bytes per cache and step, compaction moves not counted"}
@@ -423,7 +459,8 @@ def main():
                 "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
                 "config": cfg_dict(wl, {"parallelism": f"replicas x{world}" if world > 1 else "single GPU",
                                         "prefill_path": "tcgen05" if bm.last_prefill_path() == 1 else "simt-fp32",
-                                        "launch": "eager" if args.no_graph else "one CUDA graph per step, replayed",
+                                        "launch": ("eager" if args.no_graph else "one CUDA graph per step, replayed") +
+                                        (f"; {n_ranges} sample ranges on {n_ranges} streams" if n_ranges > 1 else ""),
                                         "rule": args.rule, "compaction": args.compaction,
                                         "left_pad": "none" if pads is None else
                                         f"seeded, {sum(pads)} of {wl.b * wl.s} prompt positions are padding"}),

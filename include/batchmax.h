@@ -24,7 +24,11 @@
  *     return without synchronising, except where stated.
  *   - Every function returns a bm_status_t; nothing throws, aborts or traps.
  *     On a non-BM_OK return nothing was enqueued and the cache is unchanged.
- *   - A handle is not thread-safe; distinct handles are independent.
+ *   - A handle is not thread-safe; distinct handles are independent.  One host thread may keep calls on disjoint
+ *     sample ranges of one handle in flight on different streams at the same time (the caches of different samples
+ *     are independent, and a range's scratch has its own place in the workspace) as long as max_call_samples
+ *     covers the batch (0 does) and the calls are not the *_static or *_host variants; calls that touch the same
+ *     sample must be ordered by the caller (same stream, or events).
  *   - All (sample, kv-head) caches of one (layer, sample) hold the same n, and
  *     n after a call is a function of n before, I and evict_to only, so the
  *     library mirrors n and curr_id on the host and never reads them back.

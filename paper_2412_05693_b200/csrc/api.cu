@@ -99,6 +99,7 @@ struct bm_cache {
   int32_t* kv_ids;
   int32_t* status;
   float* ws_lse;
+  float* ws_lse_own;             // the workspace's own (bm_prefill_block_static swaps ws_lse for the call)
   float* ws_new_sum;
   int32_t* left_pad = nullptr;   // [batch] device copy of the samples' padding counts (in the workspace)
   bool has_pad = false;          // some sample is left-padded
@@ -257,6 +258,7 @@ bm_status_t bm_cache_create(const bm_config_t* cfg, void* arena, size_t arena_by
   c->kv_ids = reinterpret_cast<int32_t*>(p + off);       off += rows * 4;
   if (off > need_arena) { delete c; return BM_ERR_OOM; }
   c->ws_lse = static_cast<float*>(workspace);
+  c->ws_lse_own = c->ws_lse;
   c->ws_new_sum = reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_lse_bytes(cfg));
   c->left_pad = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + ws_lse_bytes(cfg) + ws_newsum_bytes(cfg));
   c->n.assign((size_t)cfg->n_layers * cfg->batch, 0);
@@ -312,7 +314,13 @@ bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int3
   CacheView view = make_view(c, layer, sample0, nsamples, n_old, pad_active(c, layer, sample0, nsamples, pos0, I));
   BlockArgs a;
   a.q = q; a.k = k; a.v = v; a.out = out;
-  a.lse = c->ws_lse; a.new_sum = c->ws_new_sum;
+  // A range's scratch sits at its samples' own place in the workspace when the workspace covers the range there, so
+  // that calls on disjoint sample ranges may be in flight on different streams at the same time (stride block_max,
+  // whatever I is); micro-batched calls on a smaller workspace, and the static scratch, start at its beginning.
+  const bool own_ws = c->ws_lse == c->ws_lse_own;
+  const size_t s_off = (own_ws && sample0 + nsamples <= call_samples(&c->cfg)) ? (size_t)sample0 : 0;
+  a.lse = c->ws_lse + s_off * c->cfg.n_q_heads * c->cfg.block_max;
+  a.new_sum = c->ws_new_sum + s_off * c->cfg.n_kv_heads * c->cfg.block_max;
   a.I = I; a.pos0 = pos0; a.scale = c->scale;
 
   int used_tc = 0;
@@ -331,7 +339,7 @@ bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int3
   int n_new = 0;
   if (target > 0) {
     EvictArgs e;
-    e.blk_k = k; e.blk_v = v; e.new_sum = c->ws_new_sum;
+    e.blk_k = k; e.blk_v = v; e.new_sum = a.new_sum;
     e.I = I; e.pos0 = pos0; e.curr_id = pos0 + I - 1; e.target = target;
     if ((s = run_evict(c, view, e, st)) != BM_OK) return s;
     n_new = target;

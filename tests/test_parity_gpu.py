@@ -609,6 +609,48 @@ def test_cuda_graph_replay_matches_eager_launches(which):
     captured.close()
 
 
+@pytest.mark.parametrize("compaction", ["stable", "fill"])
+def test_sample_ranges_on_concurrent_streams_match_whole_batch_calls(compaction):
+    # the launch configuration of the benchmark: the batch split into sample ranges, each range's calls on a stream of
+    # its own, all in flight together; every cache must end up bit-identical to the whole-batch run
+    import torch
+    from paper_2412_05693_b200 import BatchMaxCache
+    from paper_2412_05693_b200.workloads import Inputs, schedule
+    from tests.lockstep import make_config
+    wl = WORKLOADS["cfg2"].with_(b=8, s=1536, steps=12)
+    dev = torch.device("cuda", 0)
+    inp = Inputs(wl, dev)
+    ins = [(kind, pos0, I, ev, inp.block(0, pos0, I)) for kind, pos0, I, ev in schedule(wl)]
+
+    def run(R):
+        cache = BatchMaxCache(make_config(wl, compaction=compaction))
+        outs = [torch.zeros(wl.b, I, wl.Hq, wl.d, dtype=torch.bfloat16, device=dev) for _, _, I, _, _ in ins]
+        streams = [torch.cuda.Stream() for _ in range(R)]
+        nb = wl.b // R
+        torch.cuda.synchronize()
+        for r in range(R):
+            with torch.cuda.stream(streams[r]):
+                for (kind, pos0, I, ev, (q, k, v)), o in zip(ins, outs):
+                    sl = slice(r * nb, (r + 1) * nb)
+                    if kind == "prefill":
+                        cache.prefill_block(q[sl], k[sl], v[sl], pos0, out=o[sl], evict_to=ev, sample0=r * nb)
+                    else:
+                        cache.decode_step(q[sl, 0].contiguous(), k[sl, 0].contiguous(), v[sl, 0].contiguous(),
+                                          out=o[sl, 0], evict_to=ev, sample0=r * nb)
+        torch.cuda.synchronize()
+        assert cache.status() == 0
+        state = [cache.export(0, s_, h, rows=True) for s_ in range(wl.b) for h in (0, wl.Hkv - 1)]
+        cache.close()
+        return outs, state
+
+    ref_out, ref_state = run(1)
+    for R in (2, 4):
+        outs, state = run(R)
+        assert all(torch.equal(a, b) for a, b in zip(outs, ref_out)), f"{R} ranges: outputs differ"
+        for got, want in zip(state, ref_state):
+            assert all(torch.equal(a, b) for a, b in zip(got, want)), f"{R} ranges: cache state differs"
+
+
 def test_export_import_roundtrip_resumes_identically():
     wl = tiny("ckpt", dtype="bf16", d=128, Hq=8, Hkv=2, s=192, B=64, K=48, steps=0)
     cfg = make_config(wl)
