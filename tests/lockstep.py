@@ -70,13 +70,22 @@ def check_kept(unit: UnitCache, gpu_ids: np.ndarray, target: int, stats: dict, w
 
 def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=None, check_rows_every: int = 8,
                  growth: int | None = None, sum_rtol: float | None = None, pads=None, rule: str = "average",
-                 compaction: str = "stable"):
+                 compaction: str = "stable", micro: int | None = None, micro_dec: int | None = None, arena=None,
+                 cache=None):
     """Run `calls` (default: the workload's spec schedule) on the GPU for the whole batch and on the
-    oracle for `units` = [(sample, kv_head), ...].  Returns a dict of statistics; raises on any mismatch."""
+    oracle for `units` = [(sample, kv_head), ...].  Returns a dict of statistics; raises on any mismatch.
+
+    `micro` / `micro_dec`: issue every prefill / decode call range by range (`sample0, nsamples`) with that many
+    samples per call, drawing each range's inputs on the fly -- the call pattern of batches whose prompts cannot
+    be resident at once; only the sampled units' slices of q/k/v/out are kept for the oracle.  `arena`: a caller-
+    owned byte tensor the cache is built in.  `cache`: an existing handle to run on (it is left open)."""
     dev = torch.device("cuda", device)
     inp = Inputs(wl, dev)
-    cfg = make_config(wl, device, growth, rule=rule, compaction=compaction)
-    cache = BatchMaxCache(cfg)
+    own_cache = cache is None
+    if own_cache:
+        mc = 0 if micro is None else max(micro, micro_dec or micro)
+        cfg = make_config(wl, device, growth, rule=rule, compaction=compaction, max_call_samples=min(mc, wl.b))
+        cache = BatchMaxCache(cfg, arena=arena)
     if pads is not None:                            # left-padded samples: pads[sample] padding positions
         cache.set_left_pad(pads)
     g = wl.g
@@ -86,21 +95,35 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
     sum_rtol = sum_rtol if sum_rtol is not None else (2e-3 if wl.dtype == "bf16" else 2e-4)
     calls = schedule(wl) if calls is None else calls
     from paper_2412_05693_b200 import last_prefill_path
-    for ci, (kind, pos0, I, evict_to) in enumerate(calls):
-        if kind == "evict":
-            cache.evict(evict_to, layer=layer)
-            q = k = v = out = None
-        elif kind == "recent":                      # Algorithm 3's rule; `evict_to` pairs stay
-            cache.keep_most_recent(evict_to, layer=layer)
-            q = k = v = out = None
-        else:
-            q, k, v = inp.block(layer, pos0, I)
+
+    def issue(kind, pos0, I, evict_to):
+        """One call of the schedule on the whole batch; returns {unit: (q, k, v, out)} as fp64 arrays."""
+        step = wl.b if micro is None else (micro if kind == "prefill" else (micro_dec or micro))
+        got = {}
+        for s0 in range(0, wl.b, step):
+            ns = min(step, wl.b - s0)
+            if kind == "evict":
+                cache.evict(evict_to, layer=layer, sample0=s0, nsamples=ns)
+                continue
+            if kind == "recent":                    # Algorithm 3's rule; `evict_to` pairs stay
+                cache.keep_most_recent(evict_to, layer=layer, sample0=s0, nsamples=ns)
+                continue
+            q, k, v = inp.block(layer, pos0, I, s0, ns)
             if kind == "prefill":
-                out = cache.prefill_block(q, k, v, pos0, evict_to=evict_to, layer=layer)
+                out = cache.prefill_block(q, k, v, pos0, evict_to=evict_to, layer=layer, sample0=s0)
                 stats["tc_calls"] += last_prefill_path()
             else:
                 out = cache.decode_step(q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous(),
-                                        evict_to=evict_to, layer=layer)[:, None]
+                                        evict_to=evict_to, layer=layer, sample0=s0)[:, None]
+            for (smp, kh) in oracles:
+                if s0 <= smp < s0 + ns:
+                    r = smp - s0
+                    got[(smp, kh)] = (_np(q[r, :, kh * g:(kh + 1) * g]), _np(k[r, :, kh]), _np(v[r, :, kh]),
+                                      _np(out[r, :, kh * g:(kh + 1) * g]))
+        return got
+
+    for ci, (kind, pos0, I, evict_to) in enumerate(calls):
+        got = issue(kind, pos0, I, evict_to)
         torch.cuda.synchronize(dev)
         assert cache.status() == 0
         stats["calls"] += 1
@@ -109,9 +132,9 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
             if kind == "recent":
                 unit.keep_most_recent(evict_to)
             elif kind != "evict":
-                ref = unit.process_block(_np(q[smp, :, kh * g:(kh + 1) * g]), _np(k[smp, :, kh]), _np(v[smp, :, kh]),
-                                         pos0, -1)
-                err = float(np.abs(_np(out[smp, :, kh * g:(kh + 1) * g]) - ref).max())
+                uq, uk, uv, uo = got[(smp, kh)]
+                ref = unit.process_block(uq, uk, uv, pos0, -1)
+                err = float(np.abs(uo - ref).max())
                 stats["max_out_err"] = max(stats["max_out_err"], err)
                 assert err <= tol, f"{where}: output max-abs error {err:.3e} > {tol}"
             want_rows = (ci % check_rows_every == 0) or ci == len(calls) - 1
@@ -136,5 +159,6 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
             if want_rows:
                 assert np.array_equal(_np(kr), unit.k), f"{where}: cached K rows are not the oracle's rows"
                 assert np.array_equal(_np(vr), unit.v), f"{where}: cached V rows are not the oracle's rows"
-    cache.close()
+    if own_cache:
+        cache.close()
     return stats

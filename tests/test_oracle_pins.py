@@ -347,6 +347,69 @@ def test_literal_decode_curr_id_changes_only_the_denominator():
     assert list(a[1][(s - 16) // 4]) == list(b[1][(s - 16) // 4])     # prefill part is identical
 
 
+def test_literal_decode_curr_id_flips_a_hand_counted_eviction():
+    # Algorithm 1 with limit 3 and p = 1 on a prompt of 3 tokens, head dimension 1, scale 1.  Query 0 sees pair 0
+    # alone (weight 1); query 1 is zero, so it weighs pairs 0 and 1 by 1/2 each; query 2 is 1 and the keys are
+    # ln 11, ln 2, ln 7, so its weights are 11/20, 2/20, 7/20.  Column sums: 41/20, 12/20, 7/20.
+    #   rows accumulated (Sec. 3.2's justification):  denominators 3, 2, 1 -> 41/60, 18/60, 21/60: pair 1 leaves;
+    #   the decode loop's printed curr_id = s + t - 1 = 3: denominators 4, 3, 2 -> 41/80, 16/80, 14/80: pair 2 leaves.
+    q = np.array([0.3, 0.0, 1.0, 0.7]).reshape(4, 1, 1)
+    k = np.array([math.log(11), math.log(2), math.log(7), 0.25]).reshape(4, 1)
+    v = np.array([1.0, 2.0, 3.0, 4.0]).reshape(4, 1)
+    u = UnitCache(1, 1, scale=1.0)
+    u.process_block(q[:3], k[:3], v[:3], 0)
+    np.testing.assert_allclose(u.sum_weights, [41 / 20, 12 / 20, 7 / 20], rtol=1e-14)
+    np.testing.assert_allclose(u.ave_weights(), [41 / 60, 18 / 60, 21 / 60], rtol=1e-14)
+    np.testing.assert_allclose(u.ave_weights(curr_id=3), [41 / 80, 16 / 80, 14 / 80], rtol=1e-14)
+    exact = run_algorithm1(q, k, v, 3, 3, 1, 2, scale=1.0)
+    literal = run_algorithm1(q, k, v, 3, 3, 1, 2, scale=1.0, literal_decode_curr_id=True)
+    assert list(exact[1][-1]) == [0, 2, 3]
+    assert list(literal[1][-1]) == [0, 1, 3]
+    # the decode query (0.7) then sees different pairs: softmax over keys {ln 11, ln 7, 1/4} against {ln 11, ln 2, 1/4}
+    def expected(keys, vals):
+        w = np.array([math.exp(0.7 * x) for x in keys])
+        return float((w / w.sum()) @ np.array(vals))
+    assert exact[0][3, 0, 0] == pytest.approx(expected([math.log(11), math.log(7), 0.25], [1.0, 3.0, 4.0]), rel=1e-13)
+    assert literal[0][3, 0, 0] == pytest.approx(expected([math.log(11), math.log(2), 0.25], [1.0, 2.0, 4.0]), rel=1e-13)
+
+
+def test_decode_only_compression_replayed_from_the_original_arrays():
+    # whole prompt with a full cache, ONE compression to kv_max by the average of the dense column sums, then
+    # every decode query sees the survivors of the previous call plus itself: all recomputed from the original
+    # q/k/v by masked attention written from the definition, never touching the cache structure
+    s, B, K, steps, g, d = 37, 8, 9, 11, 2, 8
+    q, k, v = rand_qkv(95, s + steps, g, d)
+    out, trace, unit = run_decode_only(q, k, v, s, B, K, steps)
+    scale = 1.0 / math.sqrt(d)
+
+    def weights(i, js):
+        w = np.zeros((g, s + steps))
+        for h in range(g):
+            logits = np.array([scale * float(q[i, h] @ k[j]) for j in js])
+            e = np.exp(logits - logits.max())
+            w[h, js] = e / e.sum()
+        return w
+
+    col = np.zeros(s + steps)
+    for i in range(s):
+        w = weights(i, list(range(i + 1)))
+        col += w.sum(axis=0)
+        np.testing.assert_allclose(out[i], w @ v, atol=1e-12)
+    ave = col[:s] / (g * (s - np.arange(s)))
+    kept = sorted(sorted(range(s), key=lambda j: (-ave[j], j))[:K])
+    assert list(trace[0]) == kept
+    for t in range(steps):
+        i = s + t
+        js = kept + [i]
+        w = weights(i, js)
+        col += w.sum(axis=0)
+        np.testing.assert_allclose(out[i], w @ v, atol=1e-12)
+        ave = {j: col[j] / (g * (i + 1 - j)) for j in js}
+        kept = sorted(sorted(js, key=lambda j: (-ave[j], j))[:K])
+        assert list(trace[t + 1]) == kept
+    np.testing.assert_allclose(unit.sum_weights, col[kept], rtol=1e-12)
+
+
 # ---------------------------------------------------------------- P7: masked-dense replay
 def test_masked_dense_replay():
     s, B, K, steps, g, d = 60, 8, 12, 7, 2, 8

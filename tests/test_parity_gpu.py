@@ -58,7 +58,7 @@ def test_cfg4_layers_are_independent():
         run_lockstep(wl, [(1, 2)], layer=layer, check_rows_every=4)
 
 
-@pytest.mark.parametrize("B,K", [CFG5_SWEEP[1], CFG5_SWEEP[3], CFG5_SWEEP[5]])
+@pytest.mark.parametrize("B,K", CFG5_SWEEP)      # all six (block, kv_max) pairs of the configuration
 def test_cfg5_large_candidate_sets(B, K):
     wl = WORKLOADS["cfg5"].with_(b=2, B=B, K=K, s=8192, steps=4)
     run_lockstep(wl, [(1, 17)], check_rows_every=4)
