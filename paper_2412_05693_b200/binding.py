@@ -181,6 +181,16 @@ def profile_pass(fn):
     return out
 
 
+def profile_read():
+    """Durations recorded since the last read, {kernel class: (total ms, launches)}; waits for them and forgets them."""
+    out = {}
+    for name, c in KERNEL_CLASSES.items():
+        ms, n = C.c_float(0), _i32(0)
+        _check(lib().bm_profile_read(c, C.byref(ms), C.byref(n)), "bm_profile_read")
+        out[name] = (float(ms.value), int(n.value))
+    return out
+
+
 def _ptr(t):
     return None if t is None else C.c_void_p(t.data_ptr())
 
