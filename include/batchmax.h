@@ -274,6 +274,10 @@ uint64_t bm_kernel_launch_count(void);
 /* Which attention implementation the last bm_prefill_block used: 0 = fp32 SIMT, 1 = tcgen05 bf16. */
 int32_t bm_last_prefill_path(void);
 const char* bm_status_string(bm_status_t s);
+/* Text of the CUDA error behind the calling thread's most recent BM_ERR_CUDA from a kernel launch ("no error" if
+ * none).  After BM_ERR_CUDA the state of the call's sample range is undefined: some of the call's kernels may have
+ * been enqueued; restore the range with bm_cache_import / bm_cache_set_len, or drop the handle. */
+const char* bm_last_cuda_error(void);
 
 #ifdef __cplusplus
 }

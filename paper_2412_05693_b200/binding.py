@@ -21,6 +21,8 @@ class BMError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
         msg = lib().bm_status_string(code).decode() if _lib is not None else ""
+        if code == 5 and _lib is not None:
+            msg += ": " + lib().bm_last_cuda_error().decode()
         super().__init__(f"{where}: {STATUS.get(code, code)} ({msg})")
 
 
@@ -67,6 +69,7 @@ SIGNATURES = {
     "bm_kernel_launch_count": (C.c_uint64, []),
     "bm_last_prefill_path": (_i32, []),
     "bm_status_string": (C.c_char_p, [_i32]),
+    "bm_last_cuda_error": (C.c_char_p, []),
 }
 
 

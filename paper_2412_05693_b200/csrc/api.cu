@@ -46,6 +46,13 @@ using namespace bm;
 
 namespace {
 
+// The CUDA error behind the most recent BM_ERR_CUDA of this thread (bm_last_cuda_error).
+thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+bm_status_t cuda_fail(cudaError_t e) {
+  g_last_cuda_error = e;
+  return BM_ERR_CUDA;
+}
+
 constexpr size_t kHeaderBytes = 1024;   // status word + room to align each of the four slabs to 256 B
 constexpr int kMaxCandidates = 12288;   // candidates of one eviction must fit one CTA's shared memory
 constexpr size_t kMaxSmem = 227 * 1024;
@@ -289,7 +296,8 @@ bm_status_t bm_cache_destroy(bm_cache_t* cache) {
 
 static bm_status_t run_evict(bm_cache* c, const CacheView& view, const EvictArgs& e, cudaStream_t st) {
   if (evict_smem_bytes(view.n_old + e.I, e.target) > kMaxSmem) return BM_ERR_CAPACITY;
-  return launch_evict(c->cfg.dtype, c->cfg.head_dim, view, e, st) == cudaSuccess ? BM_OK : BM_ERR_CUDA;
+  const cudaError_t err = launch_evict(c->cfg.dtype, c->cfg.head_dim, view, e, st);
+  return err == cudaSuccess ? BM_OK : cuda_fail(err);
 }
 
 bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int32_t nsamples, const void* q,
@@ -325,16 +333,17 @@ bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int3
 
   int used_tc = 0;
   if (c->cfg.dtype == BM_BF16 && tc_path_available()) {
-    if (launch_attn_tc(c->cfg.head_dim, view, a, st, &used_tc) != cudaSuccess) return BM_ERR_CUDA;
+    if (cudaError_t e = launch_attn_tc(c->cfg.head_dim, view, a, st, &used_tc); e != cudaSuccess) return cuda_fail(e);
   }
-  if (!used_tc && launch_attn_simt(c->cfg.dtype, c->cfg.head_dim, view, a, st) != cudaSuccess) return BM_ERR_CUDA;
+  if (!used_tc)
+    if (cudaError_t e = launch_attn_simt(c->cfg.dtype, c->cfg.head_dim, view, a, st); e != cudaSuccess) return cuda_fail(e);
   g_last_prefill_path = used_tc;
   int used_tc_score = 0;
   if (c->cfg.dtype == BM_BF16 && tc_path_available()) {
-    if (launch_score_tc(c->cfg.head_dim, view, a, st, &used_tc_score) != cudaSuccess) return BM_ERR_CUDA;
+    if (cudaError_t e = launch_score_tc(c->cfg.head_dim, view, a, st, &used_tc_score); e != cudaSuccess) return cuda_fail(e);
   }
-  if (!used_tc_score && launch_score_simt(c->cfg.dtype, c->cfg.head_dim, view, a, st) != cudaSuccess)
-    return BM_ERR_CUDA;
+  if (!used_tc_score)
+    if (cudaError_t e = launch_score_simt(c->cfg.dtype, c->cfg.head_dim, view, a, st); e != cudaSuccess) return cuda_fail(e);
 
   int n_new = 0;
   if (target > 0) {
@@ -373,7 +382,7 @@ bm_status_t bm_decode_step(bm_cache_t* c, int32_t layer, int32_t sample0, int32_
   const cudaError_t err = mma ? launch_decode_mma(c->cfg.head_dim, view, q, k, v, out, pos, c->scale, kernel_target, st)
                               : launch_decode(c->cfg.dtype, c->cfg.head_dim, view, q, k, v, out, pos, c->scale,
                                               kernel_target, st);
-  if (err != cudaSuccess) return BM_ERR_CUDA;
+  if (err != cudaSuccess) return cuda_fail(err);
   const int n_new = target >= 0 ? target : n1;
   set_mirror(c, layer, sample0, nsamples, n_new, pos);
   pad_update(c, layer, sample0, nsamples, pos, 1, n1 - n_new);
@@ -709,6 +718,8 @@ bm_status_t bm_profile_read(int32_t kernel_class, float* total_ms, int32_t* laun
   *launches = cnt;
   return ok ? BM_OK : BM_ERR_CUDA;
 }
+
+const char* bm_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda_error); }
 
 uint64_t bm_kernel_launch_count(void) { return (uint64_t)g_launch_count; }
 int32_t bm_last_prefill_path(void) { return g_last_prefill_path; }

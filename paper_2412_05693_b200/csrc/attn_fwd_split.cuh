@@ -4,8 +4,9 @@
 // warp 8 issues the MMAs and owns the tensor memory, warp 9 is the TMA producer.  The softmax of a tile is the
 // serial link between its Q.K^T and its P.V, so halving its latency shortens the whole chain; the two threads of a
 // row exchange their partial row maxima through shared memory (one named barrier per tile) and add their partial
-// row sums in the epilogue.  Two CTAs per SM; tensor memory: S 128 columns (each thread's bf16 probabilities
-// overwrite the first 32 of its own 64 logit columns) | O 128 columns.
+// row sums in the epilogue.  A thread publishes its probabilities in two halves of 32 keys, so that the first half
+// of P.V runs under the second half's exponentials.  Two CTAs per SM; tensor memory: S 128 columns (each thread's
+// bf16 probabilities overwrite the first 32 of its own 64 logit columns) | O 128 columns.
 #pragma once
 
 template <int D>
@@ -25,7 +26,7 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
   using L = SplitSmem<D>;
   constexpr int kMmaWarp = 8, kTmaWarp = 9;
   constexpr int kTmemCols = 256;
-  constexpr int B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = 3, B_SFULL = 5, B_PFULL = 6, B_ODONE = 7, B_COUNT = 8;
+  constexpr int B_QFULL = 0, B_KVFULL = 1, B_KVEMPTY = 3, B_SFULL = 5, B_PFULL = 6, B_ODONE = 7, B_PHALF = 8, B_COUNT = 9;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* sm = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   float* sEx = reinterpret_cast<float*>(sm + L::kEx);
@@ -64,6 +65,7 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
     mbar_init(&bars[B_QFULL], 1);
     mbar_init(&bars[B_SFULL], 1);
     mbar_init(&bars[B_PFULL], 256);
+    mbar_init(&bars[B_PHALF], 256);   // the first half of every thread's probabilities is published on its own
     mbar_init(&bars[B_ODONE], 1);
     for (int s = 0; s < 2; ++s) { mbar_init(&bars[B_KVFULL + s], 1); mbar_init(&bars[B_KVEMPTY + s], 1); }
     mbar_fence_init();
@@ -111,12 +113,20 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
         mma_commit(&bars[B_SFULL]);
       };
       auto issue_pv = [&](int j) {        // O += P V_j, P read from tensor memory (over S)
-        mbar_wait(&bars[B_PFULL], j & 1, abort_flag, a.status);
-        tc_fence_after();
+        // The probabilities arrive in two halves: every thread's first 32 columns (keys 0-31 and 64-95: steps 0, 1,
+        // 4, 5), then its last 32, each on a barrier of its own (one arrival per thread and key tile on either).  The
+        // first half of P.V runs under the exponentials of the second.
 #pragma unroll
-        for (int ks = 0; ks < kTileN / 16; ++ks)   // 16 keys = 2 row groups of 1024 bytes per step; P of keys 64..127 at column 64
-          mma_ts(tm_o, tm_s + (ks >> 2) * 64 + (ks & 3) * 8, dv_hi | (v_lo + ks * 128), idesc_pv,
-                 (j > 0 || ks > 0) ? 1u : 0u);
+        for (int ph = 0; ph < 2; ++ph) {
+          mbar_wait(&bars[ph ? B_PFULL : B_PHALF], j & 1, abort_flag, a.status);
+          tc_fence_after();
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int ks = (q >> 1) * 4 + ph * 2 + (q & 1);   // 16 keys per step; P of keys 64..127 sits at column 64
+            mma_ts(tm_o, tm_s + (ks >> 2) * 64 + (ks & 3) * 8, dv_hi | (v_lo + ks * 128), idesc_pv,
+                   (j > 0 || ph > 0 || q > 0) ? 1u : 0u);
+          }
+        }
         mma_commit(&bars[B_KVEMPTY + 1]);
       };
       mbar_wait(&bars[B_QFULL], 0, abort_flag, a.status);
@@ -240,6 +250,11 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
           pk[e] = pack_bf16(p0, p1);
         }
         tmem_st16(tm_s + lane_addr + c_lo + 16 * ch, pk);
+        if (ch == 0) {                              // the first half may enter P.V now
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(&bars[B_PHALF]);
+        }
       }
       l += ps0 + ps1;
       tmem_wait_st();
