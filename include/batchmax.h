@@ -23,7 +23,10 @@
  *     (a cudaStream_t passed as void*, NULL = the legacy default stream) and
  *     return without synchronising, except where stated.
  *   - Every function returns a bm_status_t; nothing throws, aborts or traps.
- *     On a non-BM_OK return nothing was enqueued and the cache is unchanged.
+ *     Every check of the arguments and of the cache state runs before the first launch: on any non-BM_OK return
+ *     other than BM_ERR_CUDA nothing was enqueued and the cache is unchanged.  BM_ERR_CUDA (a launch or copy was
+ *     refused by the runtime) can come after part of the call was enqueued: the state of the call's sample range is
+ *     then undefined (see bm_last_cuda_error).
  *   - A handle is not thread-safe; distinct handles are independent.  One host thread may keep calls on disjoint
  *     sample ranges of one handle in flight on different streams at the same time (the caches of different samples
  *     are independent, and a range's scratch has its own place in the workspace) as long as max_call_samples
@@ -114,8 +117,9 @@ bm_status_t bm_workspace_bytes(const bm_config_t* cfg /*HOST*/, size_t* bytes /*
 /* Carve `arena` (DEVICE, 256-byte aligned, >= bm_arena_bytes) into the slabs
  * K,V: [L][b][Hkv][cap][d], sum_weights: fp32 [L][b][Hkv][cap], kv_ids: int32 [L][b][Hkv][cap],
  * zero it on `cuda_stream`, and return a handle with every cache empty (n = 0, curr_id = -1).
- * `workspace` (DEVICE, 256-byte aligned, >= bm_workspace_bytes) is used by every later call; calls on
- * the same handle must therefore be stream-ordered with respect to each other.
+ * `workspace` (DEVICE, 256-byte aligned, >= bm_workspace_bytes) is used by every later call; calls that touch the
+ * same samples must be stream-ordered with respect to each other (calls on disjoint sample ranges may overlap
+ * under the conditions of the general rules above: each range has its own place in the workspace).
  * Both buffers stay owned by the caller and must outlive the handle.
  * Errors: BM_ERR_INVALID (bad config / null / misaligned), BM_ERR_OOM (a buffer is too small). */
 bm_status_t bm_cache_create(const bm_config_t* cfg /*HOST*/, void* arena /*DEVICE*/, size_t arena_bytes,
@@ -123,7 +127,7 @@ bm_status_t bm_cache_create(const bm_config_t* cfg /*HOST*/, void* arena /*DEVIC
                             bm_cache_t** out /*HOST out*/);
 bm_status_t bm_cache_destroy(bm_cache_t* cache); /* frees the host handle only */
 
-/* ---- the forward pass with a block of I inputs (Sec. 3.2; Algorithm 1 "process tokens [t0, t1-1]") ----
+/* ---- the forward pass with a block of I inputs (Sec. 3.2; the block-processing step of Algorithm 1) ----
  * For samples sample0 .. sample0+nsamples-1 of `layer`: the I queries at positions pos0 .. pos0+I-1
  * attend to all n cached pairs and to the block's own pairs at positions <= their own (causal);
  *   out = softmax(scale * q k^T) v,      sum_weights += sum_i attn_weights[i]
@@ -142,7 +146,7 @@ bm_status_t bm_prefill_block(bm_cache_t* cache, int32_t layer, int32_t sample0, 
                              const void* q, const void* k, const void* v, int32_t I, int32_t pos0,
                              void* out, int32_t evict_to, void* cuda_stream);
 
-/* ---- one decoding step (Algorithm 1 "generate token"; Sec. 3.2 "during decoding I = 1") ----
+/* ---- one decoding step (the generation step of Algorithm 1; Sec. 3.2: a block of one input) ----
  * Same as bm_prefill_block with I = 1 and pos0 = curr_id + 1, in one bandwidth-bound pass.
  *   q, out DEVICE [nsamples][Hq][d]     k, v DEVICE [nsamples][Hkv][d]
  * Needs n + 1 <= cap (the new pair is appended before an optional eviction). */
@@ -150,7 +154,7 @@ bm_status_t bm_decode_step(bm_cache_t* cache, int32_t layer, int32_t sample0, in
                            const void* q, const void* k, const void* v, void* out, int32_t evict_to,
                            void* cuda_stream);
 
-/* ---- eviction (Algorithm 1 "remove p KV pairs"; Sec. 3.2 average-attention rule) ----
+/* ---- eviction (the removal step of Algorithm 1; Sec. 3.2 average-attention rule) ----
  * For every (sample, kv-head) of the range independently:
  *   ave_weights = sum_weights / (g * (curr_id + 1 - kv_ids));
  * keep the `target` pairs that rank first under (ave_weights descending, kv_ids ascending), move them
@@ -159,11 +163,10 @@ bm_status_t bm_decode_step(bm_cache_t* cache, int32_t layer, int32_t sample0, in
 bm_status_t bm_evict(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples, int32_t target,
                      void* cuda_stream);
 
-/* ---- the rule of the extreme decoding-only comparison (Algorithm 3: "remove all but the most recent
- * KV pair") ----
+/* ---- the rule of the extreme decoding-only comparison (Algorithm 3: only the newest pair survives a cut) ----
  * Keep the `keep` most recent pairs of every cache of the range, moved to the front with their
  * sum_weights and kv_ids; n becomes keep.  No-op when n <= keep.  It exists so that the comparison arm
- * of the paper's experiments (Sec. 5, ED) runs on the same kernels and memory model as the method itself.
+ * of the paper's experiments (Sec. 4, ED) runs on the same kernels and memory model as the method itself.
  * Errors as bm_evict. */
 bm_status_t bm_keep_most_recent(bm_cache_t* cache, int32_t layer, int32_t sample0, int32_t nsamples,
                                 int32_t keep, void* cuda_stream);
@@ -174,11 +177,15 @@ bm_status_t bm_keep_most_recent(bm_cache_t* cache, int32_t layer, int32_t sample
  * library image on every GPU that loads it, instead of the workspace given to bm_cache_create.  It is
  * meant for callers that must not allocate device memory themselves: a serving loop whose memory plan is
  * frozen after start-up, a plug-in under a framework whose caching allocator owns the whole device, or a
- * thread that may not issue allocating CUDA calls.  The call itself allocates and frees nothing.
+ * thread that may not issue allocating CUDA calls.  The call itself calls no allocating routine.
  *   Limits: nsamples * Hq * I <= 1,048,576 and nsamples * Hkv * I <= 262,144, else BM_ERR_CAPACITY
- *   (nothing is enqueued).  cfg.device must be below 64.
+ *   (nothing is enqueued); the limits of bm_prefill_block apply as well (nsamples <= max_call_samples,
+ *   I <= block_max, at most 65535 caches per call).  cfg.device must be below 64.
  *   First call on a device: resolves the array's device address (cudaGetSymbolAddress with that device
- *   current).  Make that first call before starting any stream capture.
+ *   current).  Under the runtime's lazy module loading that first call is also what places the library's
+ *   device code and with it the 5 MiB array in that GPU's memory -- an allocation in all but name -- so make
+ *   it during start-up, and before starting any stream capture.  The table of resolved addresses is shared by
+ *   all handles and threads of the process (concurrent first calls store the same value).
  *   Sharing: all handles and all calls on a device use the same array, and it keeps the previous call's
  *   contents.  Nothing in it has to start from zero (every entry a call reads is written by that call
  *   first), but two calls that overlap on the GPU -- different streams, or different handles without

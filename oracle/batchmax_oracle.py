@@ -274,34 +274,85 @@ def run_north_star(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec: 
     return np.concatenate(outs, axis=0), trace, unit
 
 
-def run_algorithm1(q, k, v, s: int, kv_bar: int, p: int, max_gen: int, scale: float | None = None,
-                   literal_decode_curr_id: bool = False):
-    """Algorithm 1 as printed: first block of min(s, kv_bar) tokens; while tokens remain, remove p
-    pairs and process the next <= p tokens; then for t = 1..max_gen-1: if the cache holds kv_bar
-    pairs remove p, and process the token at position s + t - 1.
-    ``literal_decode_curr_id``: use the printed decode-time curr_id = s + t - 1 in the rule's
-    denominator (one more than the rows accumulated) instead of this build's reading."""
+def cadence_algorithm1(prompt: int, limit: int, p: int, generated: int):
+    """Algorithm 1 as a table of calls (op, first position, inputs, argument): the cache may reach ``limit`` pairs;
+    whenever it would grow past it, ``p`` pairs leave first.  The prompt's first min(prompt, limit) tokens go in
+    one block, the rest in blocks of at most ``p``; ``generated`` tokens mean ``generated - 1`` decode passes
+    (prefilling emits the first new token), each at position prompt + pass index.  Ops: "block" (argument unused),
+    "cut" (argument = pairs to keep; flagged when it happens inside the decode phase)."""
+    calls, n = [], 0
+    first = min(prompt, limit)
+    calls.append(("block", 0, first, None))
+    n, done = first, first
+    while done < prompt:
+        calls.append(("cut", 0, 0, (n - p, False)))
+        n -= p
+        take = min(p, prompt - done)
+        calls.append(("block", done, take, None))
+        n, done = n + take, done + take
+    for step in range(generated - 1):
+        if n == limit:
+            calls.append(("cut", 0, 0, (n - p, True)))
+            n -= p
+        calls.append(("block", prompt + step, 1, None))
+        n += 1
+    return calls
+
+
+def cadence_extreme_decoding(prompt: int, limit: int, generated: int, block: int | None = None):
+    """Algorithm 3 as a table of calls: the whole prompt with a full cache (in blocks of ``block`` positions when
+    given), then only the newest pair survives; each of the ``generated - 1`` decode passes appends one pair, and a
+    cache that has grown to ``limit`` pairs is cut back to its newest pair.  Ops: "block", "newest" (argument =
+    pairs to keep)."""
+    calls = []
+    block = prompt if block is None else block
+    for pos in range(0, prompt, block):
+        calls.append(("block", pos, min(block, prompt - pos), None))
+    calls.append(("newest", 0, 0, 1))
+    n = 1
+    for step in range(generated - 1):
+        calls.append(("block", prompt + step, 1, None))
+        n += 1
+        if n == limit:
+            calls.append(("newest", 0, 0, 1))
+            n = 1
+    return calls
+
+
+def run_cadence(q, k, v, calls, scale: float | None = None, decode_denominator_plus_one: bool = False):
+    """Feeds a table of calls to one cache.  Returns (outputs of every block in order, kv_ids after every block,
+    the cache, cache sizes: after every "cut" and after every decode block that follows a "newest")."""
     q = np.asarray(q, dtype=np.float64)
     unit = UnitCache(q.shape[2], q.shape[1], scale)
     outs, trace, sizes = [], [], []
-    t1 = min(s, kv_bar)
-    outs.append(unit.process_block(q[0:t1], k[0:t1], v[0:t1], 0))
-    trace.append(_trace_entry(unit))
-    while t1 < s:
-        unit.evict(len(unit) - p)
-        sizes.append(len(unit))
-        t0 = t1
-        t1 = min(s, t0 + p)
-        outs.append(unit.process_block(q[t0:t1], k[t0:t1], v[t0:t1], t0))
-        trace.append(_trace_entry(unit))
-    for t in range(1, max_gen):
-        if len(unit) == kv_bar:
-            unit.evict(len(unit) - p, curr_id=(s + t - 1) if literal_decode_curr_id else None)
+    seen_newest = False
+    for op, pos0, I, arg in calls:
+        if op == "block":
+            outs.append(unit.process_block(q[pos0:pos0 + I], k[pos0:pos0 + I], v[pos0:pos0 + I], pos0))
+            trace.append(_trace_entry(unit))
+            if seen_newest:
+                sizes.append(len(unit))
+        elif op == "cut":
+            keep, in_decode = arg
+            # the position about to be processed, not yet attended: one more than the rows accumulated
+            curr = unit.last_pos + 1 if (in_decode and decode_denominator_plus_one) else None
+            unit.evict(keep, curr_id=curr)
             sizes.append(len(unit))
-        pos = s + t - 1
-        outs.append(unit.decode_step(q[pos], k[pos], v[pos])[None])
-        trace.append(_trace_entry(unit))
+        elif op == "newest":
+            unit.keep_most_recent(arg)
+            seen_newest = True
+        else:
+            raise ValueError(op)
     return np.concatenate(outs, axis=0), trace, unit, sizes
+
+
+def run_algorithm1(q, k, v, s: int, kv_bar: int, p: int, max_gen: int, scale: float | None = None,
+                   literal_decode_curr_id: bool = False):
+    """Algorithm 1 (see :func:`cadence_algorithm1`).  ``literal_decode_curr_id``: at a removal inside the decode
+    loop use the printed decode-time curr_id (the position about to be generated, one more than the rows
+    accumulated) in the rule's denominator instead of this build's reading.
+    Returns (outputs, kv_ids after every block, cache, sizes after every removal)."""
+    return run_cadence(q, k, v, cadence_algorithm1(s, kv_bar, p, max_gen), scale, literal_decode_curr_id)
 
 
 def run_decode_only(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec: int = 1,
@@ -328,25 +379,7 @@ def run_decode_only(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec:
 
 def run_extreme_decoding(q, k, v, s: int, kv_bar: int, max_gen: int, block: int | None = None,
                          scale: float | None = None):
-    """Algorithm 3 (extreme decoding-only eviction): the whole prompt is processed with a full
-    cache (in blocks of ``block`` positions when given; the split changes nothing but rounding),
-    all but the most recent pair are removed, and for t = 1..max_gen-1 the token at position
-    s + t - 1 is processed, after which a cache that holds kv_bar pairs is cut back to its most
-    recent pair."""
-    q = np.asarray(q, dtype=np.float64)
-    unit = UnitCache(q.shape[2], q.shape[1], scale)
-    outs, sizes = [], []
-    block = s if block is None else block
-    pos = 0
-    while pos < s:
-        I = min(block, s - pos)
-        outs.append(unit.process_block(q[pos:pos + I], k[pos:pos + I], v[pos:pos + I], pos))
-        pos += I
-    unit.keep_most_recent(1)
-    for t in range(1, max_gen):
-        pos = s + t - 1
-        outs.append(unit.decode_step(q[pos], k[pos], v[pos])[None])
-        sizes.append(len(unit))
-        if len(unit) == kv_bar:
-            unit.keep_most_recent(1)
-    return np.concatenate(outs, axis=0), unit, sizes
+    """Algorithm 3, extreme decoding-only eviction (see :func:`cadence_extreme_decoding`).
+    Returns (outputs, cache, cache size after every decode pass)."""
+    out, _, unit, sizes = run_cadence(q, k, v, cadence_extreme_decoding(s, kv_bar, max_gen, block), scale)
+    return out, unit, sizes

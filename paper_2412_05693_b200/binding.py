@@ -236,6 +236,11 @@ class BatchMaxCache:
         except Exception:
             pass
 
+    def _check_out(self, out, q):
+        """The library writes `out` with q's layout: a strided view would scatter rows over other samples' slots."""
+        assert out.is_contiguous() and out.dtype == self.tdtype and out.shape == q.shape, \
+            "out must be a contiguous tensor of q's shape and dtype"
+
     # -- the four calls of the hot path -------------------------------------------------------------
     def prefill_block(self, q, k, v, pos0: int, out=None, evict_to: int = -1, layer: int = 0, sample0: int = 0,
                       stream=None):
@@ -244,6 +249,7 @@ class BatchMaxCache:
         assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and q.dtype == self.tdtype
         if out is None:
             out = self.torch.empty_like(q)
+        self._check_out(out, q)
         _check(lib().bm_prefill_block(self.h, layer, sample0, ns, _ptr(q), _ptr(k), _ptr(v), I, pos0, _ptr(out),
                                       evict_to, _stream(stream)), "bm_prefill_block")
         return out
@@ -256,6 +262,7 @@ class BatchMaxCache:
         assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and q.dtype == self.tdtype
         if out is None:
             out = self.torch.empty_like(q)
+        self._check_out(out, q)
         _check(lib().bm_prefill_block_static(self.h, layer, sample0, ns, _ptr(q), _ptr(k), _ptr(v), I, pos0,
                                              _ptr(out), evict_to, _stream(stream)), "bm_prefill_block_static")
         return out
@@ -266,6 +273,7 @@ class BatchMaxCache:
         assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and q.dtype == self.tdtype
         if out is None:
             out = self.torch.empty_like(q)
+        self._check_out(out, q)
         _check(lib().bm_decode_step(self.h, layer, sample0, ns, _ptr(q), _ptr(k), _ptr(v), _ptr(out), evict_to,
                                     _stream(stream)), "bm_decode_step")
         return out
@@ -350,9 +358,9 @@ class BatchMaxCache:
         return cut(ids), cut(sw), cut(kr), cut(vr)
 
     def import_(self, ids, sw, kr, vr, layer: int = 0, sample: int = 0, kv_head: int = 0, stream=None):
-        _check(lib().bm_cache_import(self.h, layer, sample, kv_head, _ptr(ids.contiguous()), _ptr(sw.contiguous()),
-                                     _ptr(kr.contiguous()), _ptr(vr.contiguous()), ids.shape[0], _stream(stream)),
-               "bm_cache_import")
+        ids, sw, kr, vr = (t.contiguous() for t in (ids, sw, kr, vr))   # kept alive until the call has returned
+        _check(lib().bm_cache_import(self.h, layer, sample, kv_head, _ptr(ids), _ptr(sw), _ptr(kr), _ptr(vr),
+                                     ids.shape[0], _stream(stream)), "bm_cache_import")
 
     def clear_status(self, stream=None):
         _check(lib().bm_cache_clear_status(self.h, _stream(stream)), "bm_cache_clear_status")

@@ -49,7 +49,7 @@ struct TcArgs {
 // ------------------------------------------------------------------------------------------------------
 // Score pass.  CTA = (tile of 128 candidate keys, unit).  A = the key tile (loaded once), B = the unit's query
 // tiles streamed through a ring; S^T lands in TMEM with lane = key, column = query row.  The pass is bound by
-// one exponential per visible pair, so four reducer warpgroups (one TMEM buffer each, query tiles taken round
+// one exponential per visible pair, so two reducer warpgroups (one TMEM buffer each, query tiles taken round
 // robin) keep the special-function units busy; their partial sums are added in a fixed order.
 constexpr int kScoreWG = 2;                              // reducer warpgroups == TMEM buffers of 128 columns
 constexpr int kScoreThreads = 128 * kScoreWG + 64;       // + warp 4*WG: MMA + TMEM owner, warp 4*WG+1: TMA

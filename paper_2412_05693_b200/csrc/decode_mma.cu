@@ -10,8 +10,6 @@
 // The instance for grids of at most one cache per SM (KD > 1 below) differs in how rows travel: K is loaded once and
 // kept in registers, V is staged in shared memory by TMA while the softmax phases run and read back with
 // transposing ldmatrix (standard fragment layout), and the rows behind the pair that leaves are written from there.
-#include <cstdlib>
-
 #include "evict.cuh"
 #include "tc_common.cuh"
 
@@ -664,35 +662,15 @@ int sm_count() {   // of the current device
   return count[dev];
 }
 
-int forced_threads() {   // BM_DECODE_THREADS=128|256 overrides the choice below (tuning aid)
-  static int v = -1;
-  if (v < 0) {
-    const char* e = std::getenv("BM_DECODE_THREADS");
-    v = e != nullptr ? std::atoi(e) : 0;
-  }
-  return v;
-}
-
-bool batched_allowed() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = std::getenv("BM_DECODE_BATCHED");
-    v = (e == nullptr || std::atoi(e) != 0) ? 1 : 0;
-  }
-  return v != 0;
-}
-
 template <int D, int G>
 cudaError_t launch_t(const CacheView& c, const DecodeArgs& a, cudaStream_t st) {
-  const int f = forced_threads();
   // four small CTAs per SM only pay for short caches: all four must fit into shared memory (up to about 1500 pairs
   // at g = 4), and beyond that length the larger CTA measured faster at every group size (g = 1, 4096 pairs, 2000
   // caches: 0.96 against 0.69)
   const bool four_fit = c.n_old + 1 <= 1536 && smem_layout(nullptr, D, G, c.n_old + 1, 4, nullptr) <= 56 * 1024;
-  const bool small_ctas = f == 128 || (f != 256 && four_fit && c.nsamples * c.Hkv > 2 * sm_count());
-  // a grid that leaves every CTA an SM of its own: the instance that keeps K in registers (BM_DECODE_BATCHED=0
-  // turns it off, a tuning aid)
-  const bool one_per_sm = c.nsamples * c.Hkv <= sm_count() && batched_allowed();
+  const bool small_ctas = four_fit && c.nsamples * c.Hkv > 2 * sm_count();
+  // a grid that leaves every CTA an SM of its own: the instance that keeps K in registers
+  const bool one_per_sm = c.nsamples * c.Hkv <= sm_count();
   return small_ctas ? launch_nt<D, G, 128>(c, a, st, false) : launch_nt<D, G, 256>(c, a, st, one_per_sm);
 }
 

@@ -4,7 +4,7 @@
     python -m paper_2412_05693_b200.experiments --run cfg3_ratio    # P&D vs decode-only compression, same arena
     python -m paper_2412_05693_b200.experiments --run cfg4          # 32 layers, batch that fills 120 GiB
     python -m paper_2412_05693_b200.experiments --run cfg5          # the six (block, kv_max) combinations
-    python -m paper_2412_05693_b200.experiments --run sec5          # Sec. 5's arms: BM (Algorithm 1) vs ED vs FKV
+    python -m paper_2412_05693_b200.experiments --run sec4          # Sec. 4's arms: BM (Algorithm 1) vs ED vs FKV
 
 Batches this large cannot keep their prompts resident (one block of cfg3 at b = 10072 is 63 GB of Q/K/V), so
 inputs are drawn on the fly per (layer, block, range of samples) from the seeded generator and every library
@@ -291,7 +291,7 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--run", required=True, choices=["cfg3_max", "cfg3_ratio", "cfg4", "cfg5", "sec5"])
+    ap.add_argument("--run", required=True, choices=["cfg3_max", "cfg3_ratio", "cfg4", "cfg5", "sec4"])
     ap.add_argument("--budget-gib", type=float, default=None)
     ap.add_argument("--micro", type=int, default=256)
     ap.add_argument("--layers", type=int, default=None, help="run only the first N layers (cfg4)")
@@ -326,11 +326,11 @@ def main():
         layers = range(wl.L) if args.layers is None else range(args.layers)
         res = run_arm(wl, b, "pd", args.micro, arena=arena, layers=layers, compaction=args.compaction)
         print(json.dumps({"run": "cfg4", "budget_GiB": budget / GiB, "batch": b, "pd": res}))
-    elif args.run == "sec5":
-        # The procedure of Sec. 5 on one attention layer of the larger model's shape (40 heads of 128, prompt
+    elif args.run == "sec4":
+        # The procedure of Sec. 4 on one attention layer of the larger model's shape (40 heads of 128, prompt
         # 3584, 512 tokens generated = 511 decode forwards): every arm runs at the largest batch whose caches
         # fit the same budget.  Only cache memory is modelled, so the batch ratios are those of the caches alone.
-        wl = Workload("sec5", b=1, Hq=40, Hkv=40, d=128, dtype="bf16", s=3584, B=512, K=1024,
+        wl = Workload("sec4", b=1, Hq=40, Hkv=40, d=128, dtype="bf16", s=3584, B=512, K=1024,
                       steps=args.decode_steps if args.decode_steps is not None else 511, seed=5, heavy_count=36)
         budget = int((args.budget_gib or 4.0) * GiB)
         arena = torch.empty(budget, dtype=torch.uint8, device="cuda")
@@ -338,7 +338,7 @@ def main():
         for arm, kv_bar in arms:
             b = max_batch(make_cfg(wl, 1, arm, args.micro, kv_bar=kv_bar), budget)
             res = run_arm(wl, b, arm, min(args.micro, b), arena=arena, kv_bar=kv_bar, compaction=args.compaction)
-            print(json.dumps({"run": "sec5", "budget_GiB": budget / GiB, "arm": arm, "kv_bar": kv_bar, "batch": b,
+            print(json.dumps({"run": "sec4", "budget_GiB": budget / GiB, "arm": arm, "kv_bar": kv_bar, "batch": b,
                               "result": res}), flush=True)
     else:
         for B, K in CFG5_SWEEP:

@@ -33,7 +33,7 @@ def test_algorithm1_arm_keeps_the_cache_between_kv_bar_minus_p_and_kv_bar(kv_bar
         assert n <= kv_bar                                                # the limit of Algorithm 1
         seen_full = seen_full or n == kv_bar
         if seen_full:
-            assert n >= kv_bar - p                                        # Sec. 5: |kv| >= limit - p from then on
+            assert n >= kv_bar - p                                        # Sec. 4: |kv| >= limit - p from then on
     assert make_cfg(WL, 1, "alg1", 1, kv_bar=kv_bar, p=p).cap == kv_bar
     evicts = [c for c in calls if c[0] == "evict"]
     assert all(c[3] == kv_bar - p for c in evicts)                        # p pairs removed whenever the cache is full
