@@ -278,7 +278,10 @@ bm_status_t bm_profile_read(int32_t kernel_class, float* total_ms /*HOST out*/, 
 
 /* Number of kernels this library has launched in the calling process (monotone counter). */
 uint64_t bm_kernel_launch_count(void);
-/* Which attention implementation the last bm_prefill_block used: 0 = fp32 SIMT, 1 = tcgen05 bf16. */
+/* Which attention implementation the last bm_prefill_block used: 0 = fp32 SIMT, 1 = tcgen05 bf16 (forward kernel,
+ * then the score pass), 2 = tcgen05 bf16 with forward pass and column sums in one kernel (a block of at most 128
+ * query rows, I * g, against at most four tiles of 128 keys, cached and new counted apart; no padding; not the
+ * current-query rule). */
 int32_t bm_last_prefill_path(void);
 const char* bm_status_string(bm_status_t s);
 /* Text of the CUDA error behind the calling thread's most recent BM_ERR_CUDA from a kernel launch ("no error" if

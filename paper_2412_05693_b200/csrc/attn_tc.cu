@@ -45,6 +45,7 @@ struct TcArgs {
 };
 
 #include "attn_fwd_split.cuh"
+#include "attn_onepass.cuh"
 
 // ------------------------------------------------------------------------------------------------------
 // Score pass.  CTA = (tile of 128 candidate keys, unit).  A = the key tile (loaded once), B = the unit's query
@@ -312,8 +313,31 @@ cudaError_t launch_fwd_split(const CacheView& c, const BlockArgs& a, cudaStream_
   return cudaGetLastError();
 }
 
+// the forward launch of the call in flight has taken the column sums as well: no score pass follows
+thread_local bool g_scores_done = false;
+
+// A block of at most one tile of query rows against at most four tiles of keys (cached + new), without padding and
+// under a rule that accumulates every row's weights: forward pass and column sums in one kernel (attn_onepass.cuh).
+bool onepass_applies(const CacheView& c, const BlockArgs& a) {
+  const int t_old = (c.n_old + kTileN - 1) / kTileN, t_new = (a.I + kTileN - 1) / kTileN;
+  return c.left_pad == nullptr && c.rule != 2 && a.I * c.g <= kTileM && t_old + t_new <= 4;
+}
+
+template <int D>
+cudaError_t launch_onepass(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+  using L = OnePassSmem<D>;
+  static SmemConfigured configured;
+  if (cudaError_t e = configured.ensure(attn_block_onepass<D>, (size_t)(L::kTotal)); e != cudaSuccess) return e;
+  ProfileScope prof(kAttnFwd, st);
+  attn_block_onepass<D><<<dim3(c.nsamples * c.Hkv), L::kThreads, L::kTotal, st>>>(g_maps, make_args(c, a));
+  count_launch();
+  g_scores_done = true;
+  return cudaGetLastError();
+}
+
 template <int D>
 cudaError_t launch_fwd_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+  if (onepass_applies(c, a)) return launch_onepass<D>(c, a, st);
   return c.left_pad != nullptr ? launch_fwd_split<D, true>(c, a, st) : launch_fwd_split<D, false>(c, a, st);
 }
 
@@ -362,10 +386,11 @@ bool encode_slab_rows_map(CUtensorMap* m, const void* slab, int d, int rows, int
 cudaError_t launch_attn_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used) {
   *used = 0;
   g_maps_q = nullptr;
+  g_scores_done = false;
   if (!(d == 64 || d == 128) || c.g > 8 || (kTileM % c.g) != 0) return cudaSuccess;
   if (!build_maps(d, c, a, &g_maps)) return cudaSuccess;  // fall back to the SIMT kernels
   g_maps_q = a.q;
-  *used = 1;
+  *used = onepass_applies(c, a) ? 2 : 1;
   return d == 64 ? launch_fwd_t<64>(c, a, st) : launch_fwd_t<128>(c, a, st);
 }
 
@@ -373,6 +398,7 @@ cudaError_t launch_score_tc(int d, const CacheView& c, const BlockArgs& a, cudaS
   *used = 0;
   if (g_maps_q != a.q) return cudaSuccess;  // the forward pass of this call did not take the tensor-core path
   *used = 1;
+  if (g_scores_done) return cudaSuccess;    // ... or it has taken the column sums itself
   return d == 64 ? launch_score_t<64>(c, a, st) : launch_score_t<128>(c, a, st);
 }
 

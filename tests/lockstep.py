@@ -90,7 +90,8 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
         cache.set_left_pad(pads)
     g = wl.g
     oracles = {u: UnitCache(wl.d, g, left_pad=0 if pads is None else pads[u[0]], rule=rule) for u in units}
-    stats = {"adoptions": 0, "evictions": 0, "max_out_err": 0.0, "max_sum_rel": 0.0, "calls": 0, "tc_calls": 0}
+    stats = {"adoptions": 0, "evictions": 0, "max_out_err": 0.0, "max_sum_rel": 0.0, "calls": 0, "tc_calls": 0,
+             "onepass_calls": 0}
     tol = OUT_TOL[wl.dtype]
     sum_rtol = sum_rtol if sum_rtol is not None else (2e-3 if wl.dtype == "bf16" else 2e-4)
     calls = schedule(wl) if calls is None else calls
@@ -111,7 +112,8 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
             q, k, v = inp.block(layer, pos0, I, s0, ns)
             if kind == "prefill":
                 out = cache.prefill_block(q, k, v, pos0, evict_to=evict_to, layer=layer, sample0=s0)
-                stats["tc_calls"] += last_prefill_path()
+                stats["tc_calls"] += 1 if last_prefill_path() > 0 else 0
+                stats["onepass_calls"] += 1 if last_prefill_path() == 2 else 0
             else:
                 out = cache.decode_step(q[:, 0].contiguous(), k[:, 0].contiguous(), v[:, 0].contiguous(),
                                         evict_to=evict_to, layer=layer, sample0=s0)[:, None]

@@ -154,6 +154,32 @@ def test_small_shapes(wl):
     assert st["calls"] == len(schedule(wl))
 
 
+@pytest.mark.parametrize("d,g,B,K,s", [
+    (128, 2, 64, 320, 900),      # Algorithm 1's p = 64 on a short cache: 3 cached + 1 new key tile, 128 query rows
+    (128, 1, 64, 300, 700),      # half a tile of query rows, ragged cached tile
+    (128, 4, 32, 384, 600),      # grouped heads: 32 inputs x 4 heads
+    (64, 1, 128, 256, 640),      # d = 64, a whole tile of inputs, causal part spans the tile
+    (64, 8, 16, 100, 333),       # g = 8, ragged everything
+    (128, 4, 20, 50, 171),       # rows past the block's end (80 of 128) must add nothing to the column sums
+])
+def test_short_blocks_take_forward_and_column_sums_in_one_kernel(d, g, B, K, s):
+    # one exponential per pair, logits resident in tensor memory (the single-pass variant for short caches)
+    wl = tiny(f"onepass_d{d}_g{g}_B{B}_K{K}", dtype="bf16", d=d, Hq=2 * g, Hkv=2, B=B, K=K, s=s, steps=3, b=3)
+    st = run_lockstep(wl, all_units(wl), check_rows_every=2)
+    assert st["onepass_calls"] == len([c for c in schedule(wl) if c[0] == "prefill"])
+    # the same rule with evictions made by explicit calls before each block (Algorithm 1's order), limit K + B
+    calls = []
+    n = 0
+    for kind, pos0, I, ev in schedule(wl):
+        if n + I > K + B:                     # (a decode step is a block of one input)
+            calls.append(("evict", 0, 0, K))
+            n = K
+        calls.append((kind, pos0, I, -1 if kind == "prefill" else ev))
+        n = n + I if kind == "prefill" else min(n + 1, K)
+    st = run_lockstep(wl, all_units(wl)[:3], calls=calls, growth=B, check_rows_every=2)
+    assert st["onepass_calls"] > 0
+
+
 def test_algorithm1_cadence_on_gpu():
     # Algorithm 1 as printed: limit kv_bar, remove p before each block / when full during decoding
     kv_bar, p, s, gen = 96, 32, 288, 70
