@@ -36,8 +36,10 @@ pair) is here as well, :meth:`UnitCache.keep_most_recent` and
 :func:`run_extreme_decoding`, because the library's timed comparison arm is
 checked against it.
 
-Two rules of other methods, as far as Sec. 2 describes them, can replace the
-average (``rule=`` of :class:`UnitCache`): "sum_recent" and "current_query".
+Four rules of other methods, as far as Sec. 2 describes them, can replace the
+average (``rule=`` of :class:`UnitCache`): "sum_recent" (H2O), "current_query"
+(TOVA), "window_pooled" (SnapKV) and "average_std" (RoCo); their parameters the
+paper does not give are arguments here (see :meth:`UnitCache.ranking_scores`).
 
 Parity unpinned (conventions, not derivable from the paper): the GQA sum, the
 tie direction and the denominator reading above.  Everything else is pinned by
@@ -55,12 +57,17 @@ class UnitCache:
     Sec. 3.2: ``kv_ids`` (position ids, ascending), ``sum_weights`` and the
     key/value rows themselves."""
 
-    RULES = ("average", "sum_recent", "current_query")
+    RULES = ("average", "sum_recent", "current_query", "window_pooled", "average_std")
 
     def __init__(self, d: int, g: int = 1, scale: float | None = None, left_pad: int = 0,
-                 rule: str = "average"):
+                 rule: str = "average", window: int = 32, pool: int = 7, std_share: float = 0.5):
         assert rule in self.RULES
         self.rule = rule
+        self.window = int(window)        # window_pooled: queries observed / recent pairs kept (Sec. 2, SnapKV's w)
+        self.pool = int(pool)            # window_pooled: width of the max-pooling over neighbouring positions (odd)
+        self.std_share = float(std_share)  # average_std: share of the kept pairs chosen by standard deviation
+        assert self.window >= 1 and self.pool >= 1 and self.pool % 2 == 1 and 0.0 <= self.std_share <= 1.0
+        assert not (rule == "average_std" and left_pad > 0), "average_std is defined without left padding here"
         self.d = int(d)
         self.g = int(g)
         self.left_pad = int(left_pad)  # positions 0 .. left_pad-1 of this sample are padding (Sec. 3)
@@ -69,6 +76,7 @@ class UnitCache:
         self.k = np.zeros((0, d), dtype=np.float64)
         self.v = np.zeros((0, d), dtype=np.float64)
         self.sum_weights = np.zeros(0, dtype=np.float64)
+        self.sum_sq = np.zeros(0, dtype=np.float64)   # sum of squared attention weights (average_std only)
         self.last_pos = -1            # curr_id: last position id processed
         self.evicted_mass = 0.0       # sum_weights that left with evicted pairs
         self.rows_processed = 0       # number of attention rows accumulated (queries x g)
@@ -99,13 +107,16 @@ class UnitCache:
         self.k = np.concatenate([self.k, k], axis=0)
         self.v = np.concatenate([self.v, v], axis=0)
         self.sum_weights = np.concatenate([self.sum_weights, np.zeros(I)])
+        self.sum_sq = np.concatenate([self.sum_sq, np.zeros(I)])
 
         out = np.zeros((I, self.g, self.d))
         weights = np.zeros((I, self.g, n_old + I)) if return_weights else None
         real = self.kv_ids >= self.left_pad          # padding pairs are masked for every query
         n_real_queries = 0
-        if self.rule == "current_query":
-            # only the weights of the block's last query (its g heads) count, nothing is carried over (Sec. 2)
+        # rules that look at recent queries only: the weights of the block's last query (current_query) or of its
+        # last `window` inputs (window_pooled) count, and nothing is carried over from earlier passes (Sec. 2)
+        first_counted = {"current_query": I - 1, "window_pooled": I - min(self.window, I)}.get(self.rule, 0)
+        if self.rule in ("current_query", "window_pooled"):
             self.sum_weights[:] = 0.0
         for i in range(I):
             if pos0 + i < self.left_pad:
@@ -121,8 +132,10 @@ class UnitCache:
                 w = np.exp(logits - logits.max())
                 w = w / w.sum()                      # attn_weights[i] for this head
                 out[i, h] = w @ self.v[vis]
-                if self.rule != "current_query" or i == I - 1:
+                if i >= first_counted:
                     self.sum_weights[vis] += w       # sum_weights += attn_weights[i]
+                    if self.rule == "average_std":
+                        self.sum_sq[vis] += w * w
                 if return_weights:
                     weights[i, h, vis] = w
         self.last_pos = pos0 + I - 1
@@ -154,10 +167,41 @@ class UnitCache:
           recent pairs and the pairs with the largest sum of past attention weights: the floor(target / 2) most
           recent pairs rank first (+inf), the others by their raw sum_weights.
         current_query: the rule Sec. 2 ascribes to TOVA -- the weights of the current query alone (sum_weights
-          holds nothing else under this rule, see process_block)."""
+          holds nothing else under this rule, see process_block).
+        window_pooled: the rule Sec. 2 ascribes to SnapKV -- a window of recent pairs stays (the min(window, target)
+          most recent candidates, +inf); the others are ranked by the attention weights summed over the last
+          `window` queries (what sum_weights holds under this rule), each replaced by the maximum over the `pool`
+          neighbouring candidates centred on it (neighbours in cache order, the window excluded), so that kept
+          positions come in runs rather than isolated.  Pooling by maximum and the two widths are this build's
+          parameters: the paper names the pooling layer without describing it.
+        average_std: the rule Sec. 2 / Sec. 3.2 ascribe to RoCo -- the kept pairs are split between the pairs whose
+          attention weights have the largest standard deviation, floor(std_share * target) of them (+inf; ties to
+          the lower position), and the largest average weights among the rest.  The standard deviation is over the
+          g * (curr_id + 1 - kv_ids) weights the pair has received: sqrt(E[w^2] - E[w]^2).  The share is this
+          build's parameter."""
         if self.rule == "average":
             return self.ave_weights(curr_id)
+        if self.rule == "average_std":
+            ave = self.ave_weights(curr_id)
+            curr = self.last_pos if curr_id is None else curr_id
+            cnt = self.g * (curr + 1 - self.kv_ids)
+            std = np.sqrt(np.maximum(self.sum_sq / cnt - ave * ave, 0.0))
+            n_std = int(math.floor(self.std_share * int(target) + 1e-9))
+            protected = np.lexsort((self.kv_ids, -std))[:n_std]
+            score = ave.copy()
+            score[protected] = np.inf
+            return score
         score = self.sum_weights.copy()
+        if self.rule == "window_pooled":
+            n = len(self)
+            keep_recent = min(self.window, int(target))
+            body = n - keep_recent                     # candidates outside the window of recent pairs
+            half = self.pool // 2
+            pooled = np.array([score[max(0, j - half):min(body, j + half + 1)].max() for j in range(body)])
+            score[:body] = pooled
+            score[body:] = np.inf
+            score[self.kv_ids < self.left_pad] = 0.0
+            return score
         if self.rule == "sum_recent":
             window = int(target) // 2
             if window > 0:
@@ -205,6 +249,7 @@ class UnitCache:
         self.k = self.k[keep]
         self.v = self.v[keep]
         self.sum_weights = self.sum_weights[keep]
+        self.sum_sq = self.sum_sq[keep]
         self.last_eviction = snap
         return snap
 
@@ -223,6 +268,7 @@ class UnitCache:
         self.k = self.k[first:]
         self.v = self.v[first:]
         self.sum_weights = self.sum_weights[first:]
+        self.sum_sq = self.sum_sq[first:]
 
 
 # ---------------------------------------------------------------------- plain definition
@@ -251,7 +297,8 @@ def _trace_entry(unit: UnitCache):
 
 
 def run_north_star(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec: int = 1,
-                   g: int | None = None, scale: float | None = None, left_pad: int = 0, rule: str = "average"):
+                   g: int | None = None, scale: float | None = None, left_pad: int = 0, rule: str = "average",
+                   **rule_params):
     """Blocks of ``block`` prompt tokens (ragged tail allowed), the cache cut back to ``kv_max``
     after every block; then ``steps`` decode steps, cut back to ``kv_max`` whenever the cache
     has grown to ``kv_max + p_dec``.   q: (s+steps, g, d); k, v: (s+steps, d); the first
@@ -259,7 +306,7 @@ def run_north_star(q, k, v, s: int, block: int, kv_max: int, steps: int, p_dec: 
     Returns (outputs (s+steps, g, d), trace of kv_ids after every call, unit)."""
     q = np.asarray(q, dtype=np.float64)
     g = q.shape[1] if g is None else g
-    unit = UnitCache(q.shape[2], g, scale, left_pad, rule)
+    unit = UnitCache(q.shape[2], g, scale, left_pad, rule, **rule_params)
     outs, trace = [], []
     pos = 0
     while pos < s:

@@ -681,6 +681,93 @@ def test_alternative_rules_against_a_replay_from_the_original_arrays(rule):
         cached = kept
 
 
+@pytest.mark.parametrize("w,pool", [(3, 1), (4, 3), (20, 5), (2, 7)])
+def test_window_pooled_rule_against_a_replay_from_the_original_arrays(w, pool):
+    # SnapKV as Sec. 2 describes it: scores = attention weights summed over the last w queries of the pass, pooled
+    # over neighbouring positions, a window of recent pairs always kept.  Re-derived from the trace and the original
+    # arrays, with the pooling written as a plain loop over the candidates' order.
+    s, B, K, steps, g, d = 44, 9, 10, 5, 2, 4
+    q, k, v = rand_qkv(73, s + steps, g, d)
+    out, trace, unit = run_north_star(q, k, v, s, B, K, steps, rule="window_pooled", window=w, pool=pool)
+    scale = 1.0 / math.sqrt(d)
+    cached = []
+    calls = [(p0, min(B, s - p0)) for p0 in range(0, s, B)] + [(s + t, 1) for t in range(steps)]
+    for call, (p0, I) in enumerate(calls):
+        cand = list(cached) + list(range(p0, p0 + I))
+        sums = {j: 0.0 for j in cand}
+        for i in range(I - min(w, I), I):
+            qi = p0 + i
+            vis = list(cached) + list(range(p0, qi + 1))
+            for (_, h), wt in replay_weights(q, k, [vis], [qi], scale).items():
+                for j, wj in wt.items():
+                    sums[j] += wj
+        if len(cand) > K:
+            recent = cand[len(cand) - min(w, K):]
+            body = cand[:len(cand) - len(recent)]
+            pooled = {}
+            for x, j in enumerate(body):
+                lo, hi = max(0, x - pool // 2), min(len(body), x + pool // 2 + 1)
+                pooled[j] = max(sums[body[y]] for y in range(lo, hi))
+            rest = sorted(body, key=lambda j: (-pooled[j], j))
+            kept = sorted(recent + rest[:K - len(recent)])
+        else:
+            kept = cand
+        assert kept == list(trace[call]), f"call {call}"
+        cached = kept
+
+
+@pytest.mark.parametrize("share,g", [(0.0, 1), (0.5, 2), (0.3, 1), (1.0, 2)])
+def test_average_std_rule_against_a_replay_from_the_original_arrays(share, g):
+    # RoCo as Sec. 2 / Sec. 3.2 describe it: part of the kept pairs by the standard deviation of their attention
+    # weights, the rest by their average.  The replay keeps, per pair, the plain list of every weight it received.
+    s, B, K, steps, d = 40, 8, 9, 6, 4
+    q, k, v = rand_qkv(79, s + steps, g, d)
+    out, trace, unit = run_north_star(q, k, v, s, B, K, steps, rule="average_std", std_share=share)
+    scale = 1.0 / math.sqrt(d)
+    cached, got = [], {}
+    calls = [(p0, min(B, s - p0)) for p0 in range(0, s, B)] + [(s + t, 1) for t in range(steps)]
+    for call, (p0, I) in enumerate(calls):
+        cand = list(cached) + list(range(p0, p0 + I))
+        for i in range(I):
+            qi = p0 + i
+            vis = list(cached) + list(range(p0, qi + 1))
+            for (_, h), wt in replay_weights(q, k, [vis], [qi], scale).items():
+                for j, wj in wt.items():
+                    got.setdefault(j, []).append(wj)
+        if len(cand) > K:
+            assert all(len(got[j]) == g * (p0 + I - j) for j in cand)      # one weight per later-or-equal query and head
+            std = {j: float(np.std(got[j])) for j in cand}                 # population standard deviation
+            ave = {j: float(np.mean(got[j])) for j in cand}
+            n_std = int(math.floor(share * K + 1e-9))
+            protected = sorted(cand, key=lambda j: (-std[j], j))[:n_std]
+            rest = sorted([j for j in cand if j not in protected], key=lambda j: (-ave[j], j))
+            kept = sorted(protected + rest[:K - n_std])
+        else:
+            kept = cand
+        assert kept == list(trace[call]), f"call {call}"
+        got = {j: got[j] for j in kept}
+        cached = kept
+    if share == 0.0:      # no pair chosen by deviation: the method's own rule
+        _, trace_ave, _ = run_north_star(q, k, v, s, B, K, steps)
+        assert all(list(a) == list(b) for a, b in zip(trace, trace_ave))
+
+
+def test_window_pooled_with_window_one_and_no_pooling_is_the_current_query_rule_plus_its_newest_pair():
+    # w = 1, pool = 1: scores are the last query's weights (as under current_query); the one difference is that
+    # the newest pair is never a candidate for removal
+    s, B, K, g, d = 30, 6, 5, 1, 4
+    q, k, v = rand_qkv(83, s, g, d)
+    u = UnitCache(d, g, rule="window_pooled", window=1, pool=1)
+    u2 = UnitCache(d, g, rule="current_query")
+    for p0 in range(0, s, B):
+        u.process_block(q[p0:p0 + B], k[p0:p0 + B], v[p0:p0 + B], p0)
+        u2.process_block(q[p0:p0 + B], k[p0:p0 + B], v[p0:p0 + B], p0)
+        np.testing.assert_allclose(u.sum_weights, u2.sum_weights, rtol=1e-14)
+        u.evict(K)
+        assert u.kv_ids[-1] == p0 + B - 1
+        u2.evict(K, kept_ids=u.kv_ids)
+
+
 def test_sum_recent_keeps_its_window_and_current_query_forgets():
     g, d = 1, 4
     q, k, v = rand_qkv(67, 30, g, d)
