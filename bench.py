@@ -55,8 +55,10 @@ def parse_args(argv=None):
     ap.add_argument("--prompt", type=int, default=None, help="override the workload's prompt length")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps")
     ap.add_argument("--layers", type=int, default=None, help="run only the first N layers (cfg4_max)")
-    ap.add_argument("--rule", default="average", choices=["average", "sum_recent", "current_query"],
-                    help="eviction rule: the paper's average attention, or one of the rules of Sec. 2")
+    ap.add_argument("--rule", default="average",
+                    choices=["average", "sum_recent", "current_query", "window_pooled", "average_std"],
+                    help="eviction rule: the paper's average attention, or one of the rules of Sec. 2 (H2O, TOVA, SnapKV "
+                         "with window 32 / pool 7, RoCo with half of the kept pairs by standard deviation)")
     ap.add_argument("--compaction", default="stable", choices=["stable", "fill"],
                     help="stable: a cache's rows stay in position order (rows behind a pair that leaves move up); "
                          "fill: unordered rows, pairs that stay never move (same kept sets and outputs)")

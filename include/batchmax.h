@@ -68,8 +68,23 @@ typedef enum { BM_F32 = 0, BM_BF16 = 1 } bm_dtype_t;
  *   BM_RULE_CURRENT_QUERY (TOVA): pairs are ranked by the attention weights of the current query alone --
  *                         sum_weights is overwritten (not accumulated) with the weights of the block's last
  *                         query, or of the decode step's query, summed over the group's heads.
- * Ties keep the lower position under every rule. */
-typedef enum { BM_RULE_AVERAGE = 0, BM_RULE_SUM_RECENT = 1, BM_RULE_CURRENT_QUERY = 2 } bm_rule_t;
+ *   BM_RULE_WINDOW_POOLED (SnapKV): a window of recent pairs stays -- the min(window, target) most recent candidates --
+ *                         and the others are ranked by the attention weights summed over the last `window` queries:
+ *                         sum_weights is overwritten by every pass with the column sums over its last min(window, I)
+ *                         inputs (a decode step: its one query), and at an eviction every score is replaced by the
+ *                         maximum over the `pool` neighbouring candidates centred on it (cache order, the window left
+ *                         out), so that kept positions come in runs.  Pooling by maximum and both widths are this
+ *                         library's parameters: the paper names the pooling layer without describing it.
+ *   BM_RULE_AVERAGE_STD   (RoCo; also Sec. 3.2, last paragraph): the kept pairs are split between the
+ *                         floor(target * std_share_permille / 1000) pairs whose attention weights have the largest
+ *                         standard deviation, sqrt(E[w^2] - E[w]^2) over the g * (curr_id + 1 - kv_ids) weights a pair
+ *                         has received, and the largest ave_weights among the rest.  The cache keeps one more fp32
+ *                         per row (the sum of squared weights: 4 more bytes per row in the memory model).  Not
+ *                         available with left padding or through bm_prefill_block_static.
+ * Ties keep the lower position under every rule.  The last two rank by the rows' position order and need
+ * BM_COMPACT_STABLE. */
+typedef enum { BM_RULE_AVERAGE = 0, BM_RULE_SUM_RECENT = 1, BM_RULE_CURRENT_QUERY = 2, BM_RULE_WINDOW_POOLED = 3,
+               BM_RULE_AVERAGE_STD = 4 } bm_rule_t;
 
 /* What "remove pairs" does to the rows of a cache.  Attention, the scores and the kept sets do not depend on the
  * order of a cache's rows; only the work of removing does.
@@ -98,12 +113,15 @@ typedef struct {
   int32_t max_call_samples; /* largest nsamples of any call (sizes the workspace); 0 -> batch */
   int32_t rule;             /* bm_rule_t: what pairs are ranked by at an eviction; 0 = the paper's  */
   int32_t compaction;       /* bm_compaction_t: 0 = rows stay in position order                     */
+  int32_t window;           /* BM_RULE_WINDOW_POOLED: queries observed = recent pairs kept, >= 1     */
+  int32_t pool;             /* BM_RULE_WINDOW_POOLED: width of the max-pooling, odd, 1 .. 255 (1 = none) */
+  int32_t std_share_permille; /* BM_RULE_AVERAGE_STD: share of the kept pairs chosen by deviation, 0 .. 1000 */
 } bm_config_t;
 
 /* ---- cache layout, allocator and memory model (Sec. 1: batch size under a fixed memory budget) ----
  * Per sample the arena holds, for every layer and kv-head, cap = K + growth rows of:
  * key (d elements), value (d elements), sum_weights (fp32) and kv_ids (int32):
- *     bytes_per_sample = L * Hkv * cap * (2 * d * elem_size + 8).
+ *     bytes_per_sample = L * Hkv * cap * (2 * d * elem_size + 8)      (+ 4 per row under BM_RULE_AVERAGE_STD).
  * The arena adds a fixed 1024-byte header (status word, alignment of the four slabs). */
 bm_status_t bm_cache_bytes_per_sample(const bm_config_t* cfg /*HOST*/, size_t* bytes /*HOST out*/);
 /* Arena size for cfg->batch samples. */
@@ -246,6 +264,12 @@ bm_status_t bm_cache_import(bm_cache_t* cache, int32_t layer, int32_t sample, in
                             const int32_t* kv_ids /*HOST*/, const float* sum_weights /*HOST*/,
                             const void* k_rows /*HOST*/, const void* v_rows /*HOST*/, int32_t n,
                             void* cuda_stream);
+/* The same for the sums of squared weights a cache keeps under BM_RULE_AVERAGE_STD (n entries, n = the sample's
+ * mirrored length); BM_ERR_INVALID under any other rule.  Both synchronise cuda_stream. */
+bm_status_t bm_cache_export_sum_sq(bm_cache_t* cache, int32_t layer, int32_t sample, int32_t kv_head,
+                                   float* sum_sq /*HOST out*/, void* cuda_stream);
+bm_status_t bm_cache_import_sum_sq(bm_cache_t* cache, int32_t layer, int32_t sample, int32_t kv_head,
+                                   const float* sum_sq /*HOST*/, void* cuda_stream);
 /* Set the mirrored n (0 <= n <= cap) and curr_id of one (layer, sample) when restoring a checkpoint. */
 bm_status_t bm_cache_set_len(bm_cache_t* cache, int32_t layer, int32_t sample, int32_t n, int32_t curr_id);
 /* Synchronise cuda_stream and read the device status word: BM_OK, or BM_ERR_TIMEOUT if a kernel gave

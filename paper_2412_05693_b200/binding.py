@@ -31,10 +31,12 @@ class bm_config_t(C.Structure):
                 ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("kv_max", C.c_int32),
                 ("block_max", C.c_int32), ("growth", C.c_int32), ("dtype", C.c_int32),
                 ("softmax_scale", C.c_float), ("device", C.c_int32), ("max_call_samples", C.c_int32),
-                ("rule", C.c_int32), ("compaction", C.c_int32)]
+                ("rule", C.c_int32), ("compaction", C.c_int32), ("window", C.c_int32), ("pool", C.c_int32),
+                ("std_share_permille", C.c_int32)]
 
 
 _lib = None
+RULES = {"average": 0, "sum_recent": 1, "current_query": 2, "window_pooled": 3, "average_std": 4}
 
 # name -> (restype, argtypes); every symbol include/batchmax.h declares
 _vp, _i32, _sz = C.c_void_p, C.c_int32, C.c_size_t
@@ -61,6 +63,8 @@ SIGNATURES = {
     "bm_cache_export": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, C.POINTER(_i32), _vp]),
     "bm_cache_import": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _i32, _vp]),
     "bm_cache_set_len": (_i32, [_vp, _i32, _i32, _i32, _i32]),
+    "bm_cache_export_sum_sq": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp]),
+    "bm_cache_import_sum_sq": (_i32, [_vp, _i32, _i32, _i32, _vp, _vp]),
     "bm_cache_status": (_i32, [_vp, C.POINTER(_i32), _vp]),
     "bm_cache_clear_status": (_i32, [_vp, _vp]),
     "bm_selftest_wait_timeout": (_i32, [_vp, _vp]),
@@ -107,15 +111,18 @@ class Config:
     softmax_scale: float = 0.0
     device: int = 0
     max_call_samples: int = 0
-    rule: str = "average"        # "average" (the paper's) | "sum_recent" | "current_query"
+    rule: str = "average"        # "average" (the paper's) | "sum_recent" | "current_query" | "window_pooled" | "average_std"
     compaction: str = "stable"   # "stable": rows stay in position order | "fill": unordered, kept pairs never move
+    window: int = 32             # window_pooled: queries observed = recent pairs kept
+    pool: int = 7                # window_pooled: width of the max-pooling (odd)
+    std_share: float = 0.5       # average_std: share of the kept pairs chosen by standard deviation
 
     def c(self) -> bm_config_t:
         return bm_config_t(self.batch, self.n_layers, self.n_q_heads, self.n_kv_heads, self.head_dim, self.kv_max,
                            self.block_max, self.growth, BM_BF16 if self.dtype == "bf16" else BM_F32,
                            self.softmax_scale, self.device, self.max_call_samples,
-                           {"average": 0, "sum_recent": 1, "current_query": 2}[self.rule],
-                           {"stable": 0, "fill": 1}[self.compaction])
+                           RULES[self.rule], {"stable": 0, "fill": 1}[self.compaction], self.window, self.pool,
+                           int(round(self.std_share * 1000)))
 
     @property
     def cap(self) -> int:
@@ -361,6 +368,19 @@ class BatchMaxCache:
         ids, sw, kr, vr = (t.contiguous() for t in (ids, sw, kr, vr))   # kept alive until the call has returned
         _check(lib().bm_cache_import(self.h, layer, sample, kv_head, _ptr(ids), _ptr(sw), _ptr(kr), _ptr(vr),
                                      ids.shape[0], _stream(stream)), "bm_cache_import")
+
+    def export_sum_sq(self, layer: int = 0, sample: int = 0, kv_head: int = 0, stream=None):
+        """Sums of squared attention weights of one cache (rule "average_std"), float32[n] on the CPU."""
+        n0, _ = self.length(layer, sample)
+        sq = self.torch.empty(max(n0, 1), dtype=self.torch.float32)
+        _check(lib().bm_cache_export_sum_sq(self.h, layer, sample, kv_head, _ptr(sq), _stream(stream)),
+               "bm_cache_export_sum_sq")
+        return sq[:n0]
+
+    def import_sum_sq(self, sq, layer: int = 0, sample: int = 0, kv_head: int = 0, stream=None):
+        sq = sq.contiguous()
+        _check(lib().bm_cache_import_sum_sq(self.h, layer, sample, kv_head, _ptr(sq), _stream(stream)),
+               "bm_cache_import_sum_sq")
 
     def clear_status(self, stream=None):
         _check(lib().bm_cache_clear_status(self.h, _stream(stream)), "bm_cache_clear_status")

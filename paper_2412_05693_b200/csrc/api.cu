@@ -72,15 +72,20 @@ bool config_ok(const bm_config_t* c, bool need_batch) {
   if (!(c->dtype == BM_F32 || c->dtype == BM_BF16)) return false;
   if (!(c->softmax_scale >= 0.f) || std::isinf(c->softmax_scale)) return false;
   if (c->device < 0 || c->max_call_samples < 0) return false;
-  if (c->rule < 0 || c->rule > 2) return false;
+  if (c->rule < 0 || c->rule > 4) return false;
   if (c->compaction < 0 || c->compaction > 1) return false;
+  if (c->rule >= 3 && c->compaction != BM_COMPACT_STABLE) return false;   // both rank by the rows' position order
+  if (c->rule == BM_RULE_WINDOW_POOLED && (c->window < 1 || c->pool < 1 || c->pool % 2 == 0 || c->pool > 255)) return false;
+  if (c->rule == BM_RULE_AVERAGE_STD && (c->std_share_permille < 0 || c->std_share_permille > 1000)) return false;
   if ((long long)c->kv_max + c->growth > (1 << 24)) return false;
   return true;
 }
 
 size_t per_sample_bytes(const bm_config_t* c) {
   const size_t cap = (size_t)c->kv_max + c->growth;
-  return (size_t)c->n_layers * c->n_kv_heads * cap * (2 * (size_t)c->head_dim * elem_size(c->dtype) + 8);
+  // key row, value row, sum_weights, kv_ids; under BM_RULE_AVERAGE_STD also the sum of squared weights
+  const size_t per_row = 2 * (size_t)c->head_dim * elem_size(c->dtype) + 8 + (c->rule == BM_RULE_AVERAGE_STD ? 4 : 0);
+  return (size_t)c->n_layers * c->n_kv_heads * cap * per_row;
 }
 
 int call_samples(const bm_config_t* c) { return c->max_call_samples > 0 ? c->max_call_samples : c->batch; }
@@ -92,6 +97,7 @@ size_t ws_newsum_bytes(const bm_config_t* c) {
   return align_up(sizeof(float) * (size_t)call_samples(c) * c->n_kv_heads * c->block_max, 256);
 }
 size_t ws_pad_bytes(const bm_config_t* c) { return align_up(sizeof(int32_t) * (size_t)c->batch, 256); }
+size_t ws_newsq_bytes(const bm_config_t* c) { return c->rule == BM_RULE_AVERAGE_STD ? ws_newsum_bytes(c) : 0; }
 
 }  // namespace
 
@@ -103,11 +109,13 @@ struct bm_cache {
   char* k_slab;
   char* v_slab;
   float* sum_weights;
+  float* sum_sq = nullptr;       // BM_RULE_AVERAGE_STD only
   int32_t* kv_ids;
   int32_t* status;
   float* ws_lse;
   float* ws_lse_own;             // the workspace's own (bm_prefill_block_static swaps ws_lse for the call)
   float* ws_new_sum;
+  float* ws_new_sq = nullptr;    // BM_RULE_AVERAGE_STD only
   int32_t* left_pad = nullptr;   // [batch] device copy of the samples' padding counts (in the workspace)
   bool has_pad = false;          // some sample is left-padded
   // Padding leaves first at every eviction (under every rule), so how many padding pairs a sample's caches still
@@ -196,6 +204,8 @@ CacheView make_view(const bm_cache* c, int layer, int sample0, int nsamples, int
   v.left_pad = (c->has_pad && with_pad) ? c->left_pad + sample0 : nullptr;
   v.rule = c->cfg.rule;
   v.fill = c->cfg.compaction == BM_COMPACT_FILL ? 1 : 0;
+  v.sum_sq = c->sum_sq != nullptr ? c->sum_sq + row0 : nullptr;
+  v.window = c->cfg.window; v.pool = c->cfg.pool; v.std_permille = c->cfg.std_share_permille;
   v.moved = c->count_moves ? reinterpret_cast<unsigned long long*>(c->status + 16) : nullptr;
   return v;
 }
@@ -231,7 +241,7 @@ bm_status_t bm_max_batch(const bm_config_t* cfg, size_t hbm_budget_bytes, int32_
 
 bm_status_t bm_workspace_bytes(const bm_config_t* cfg, size_t* bytes) {
   if (!config_ok(cfg, true) || bytes == nullptr) return BM_ERR_INVALID;
-  *bytes = ws_lse_bytes(cfg) + ws_newsum_bytes(cfg) + ws_pad_bytes(cfg);
+  *bytes = ws_lse_bytes(cfg) + ws_newsum_bytes(cfg) + ws_pad_bytes(cfg) + ws_newsq_bytes(cfg);
   return BM_OK;
 }
 
@@ -263,11 +273,17 @@ bm_status_t bm_cache_create(const bm_config_t* cfg, void* arena, size_t arena_by
   c->v_slab = p + off;                                   off = align_up(off + slab, 256);
   c->sum_weights = reinterpret_cast<float*>(p + off);    off = align_up(off + rows * 4, 256);
   c->kv_ids = reinterpret_cast<int32_t*>(p + off);       off += rows * 4;
+  if (cfg->rule == BM_RULE_AVERAGE_STD) {   // a fifth slab of 4-byte entries right behind the fourth
+    c->sum_sq = reinterpret_cast<float*>(p + off);       off += rows * 4;
+  }
   if (off > need_arena) { delete c; return BM_ERR_OOM; }
   c->ws_lse = static_cast<float*>(workspace);
   c->ws_lse_own = c->ws_lse;
   c->ws_new_sum = reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_lse_bytes(cfg));
   c->left_pad = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + ws_lse_bytes(cfg) + ws_newsum_bytes(cfg));
+  if (cfg->rule == BM_RULE_AVERAGE_STD)
+    c->ws_new_sq = reinterpret_cast<float*>(static_cast<char*>(workspace) + ws_lse_bytes(cfg) + ws_newsum_bytes(cfg) +
+                                            ws_pad_bytes(cfg));
   c->n.assign((size_t)cfg->n_layers * cfg->batch, 0);
   c->curr_id.assign((size_t)cfg->n_layers * cfg->batch, -1);
   // Unwritten rows are read as zero-weight padding by the tiled kernels, so they must hold finite values.
@@ -329,6 +345,7 @@ bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int3
   const size_t s_off = (own_ws && sample0 + nsamples <= call_samples(&c->cfg)) ? (size_t)sample0 : 0;
   a.lse = c->ws_lse + s_off * c->cfg.n_q_heads * c->cfg.block_max;
   a.new_sum = c->ws_new_sum + s_off * c->cfg.n_kv_heads * c->cfg.block_max;
+  a.new_sq = c->ws_new_sq != nullptr ? c->ws_new_sq + s_off * c->cfg.n_kv_heads * c->cfg.block_max : nullptr;
   a.I = I; a.pos0 = pos0; a.scale = c->scale;
 
   int used_tc = 0;
@@ -348,7 +365,7 @@ bm_status_t bm_prefill_block(bm_cache_t* c, int32_t layer, int32_t sample0, int3
   int n_new = 0;
   if (target > 0) {
     EvictArgs e;
-    e.blk_k = k; e.blk_v = v; e.new_sum = a.new_sum;
+    e.blk_k = k; e.blk_v = v; e.new_sum = a.new_sum; e.new_sq = a.new_sq;
     e.I = I; e.pos0 = pos0; e.curr_id = pos0 + I - 1; e.target = target;
     if ((s = run_evict(c, view, e, st)) != BM_OK) return s;
     n_new = target;
@@ -560,6 +577,7 @@ bm_status_t bm_cache_set_left_pad(bm_cache_t* c, const int32_t* pads, void* cuda
     if (v != 0) return BM_ERR_STATE;
   for (int v : c->curr_id)
     if (v != -1) return BM_ERR_STATE;
+  if (c->cfg.rule == BM_RULE_AVERAGE_STD) return BM_ERR_INVALID;   // that rule is defined without padding here
   bool any = false;
   if (pads != nullptr)
     for (int s = 0; s < c->cfg.batch; ++s) {
@@ -666,6 +684,37 @@ bm_status_t bm_cache_import(bm_cache_t* c, int32_t layer, int32_t sample, int32_
   return ok ? BM_OK : BM_ERR_CUDA;
 }
 
+bm_status_t bm_cache_export_sum_sq(bm_cache_t* c, int32_t layer, int32_t sample, int32_t kv_head, float* sum_sq,
+                                   void* cuda_stream) {
+  size_t row0 = 0;
+  bm_status_t s = unit_offsets(c, layer, sample, kv_head, &row0);
+  if (s != BM_OK) return s;
+  if (sum_sq == nullptr || c->sum_sq == nullptr) return BM_ERR_INVALID;
+  if ((s = set_device(c)) != BM_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int cnt = c->n[(size_t)layer * c->cfg.batch + sample];
+  bool ok = true;
+  if (cnt > 0) ok &= cudaMemcpyAsync(sum_sq, c->sum_sq + row0, 4 * (size_t)cnt, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok &= cudaStreamSynchronize(st) == cudaSuccess;
+  return ok ? BM_OK : BM_ERR_CUDA;
+}
+
+bm_status_t bm_cache_import_sum_sq(bm_cache_t* c, int32_t layer, int32_t sample, int32_t kv_head, const float* sum_sq,
+                                   void* cuda_stream) {
+  size_t row0 = 0;
+  bm_status_t s = unit_offsets(c, layer, sample, kv_head, &row0);
+  if (s != BM_OK) return s;
+  if (sum_sq == nullptr || c->sum_sq == nullptr) return BM_ERR_INVALID;
+  if ((s = set_device(c)) != BM_OK) return s;
+  ++c->dev_calls;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int cnt = c->n[(size_t)layer * c->cfg.batch + sample];
+  bool ok = true;
+  if (cnt > 0) ok &= cudaMemcpyAsync(c->sum_sq + row0, sum_sq, 4 * (size_t)cnt, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaStreamSynchronize(st) == cudaSuccess;
+  return ok ? BM_OK : BM_ERR_CUDA;
+}
+
 bm_status_t bm_cache_status(bm_cache_t* c, int32_t* device_status, void* cuda_stream) {
   if (c == nullptr || device_status == nullptr) return BM_ERR_INVALID;
   bm_status_t s = set_device(c);
@@ -761,6 +810,7 @@ extern "C" bm_status_t bm_prefill_block_static(bm_cache_t* c, int32_t layer, int
                                                int32_t pos0, void* out, int32_t evict_to, void* cuda_stream) {
   if (c == nullptr) return BM_ERR_INVALID;
   if (nsamples < 1 || I < 1) return BM_ERR_INVALID;
+  if (c->cfg.rule == BM_RULE_AVERAGE_STD) return BM_ERR_INVALID;   // its second accumulator has no room in the array
   const int dev = c->cfg.device;
   if (dev < 0 || dev >= kMaxDevices) return BM_ERR_INVALID;
   if ((size_t)nsamples * c->cfg.n_q_heads * (size_t)I > kStaticLseFloats ||

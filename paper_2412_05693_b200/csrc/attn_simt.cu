@@ -197,28 +197,31 @@ __global__ void __launch_bounds__(kThreads) score_simt(CacheView c, BlockArgs a)
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
 
   load_tile<T, D>(sK, tid, [&](int r) { return key_row_ptr<T, D>(c, c.k_slab, a.k, unit, smp, kh, a.I, j0 + r); });
-  float col[4] = {0.f, 0.f, 0.f, 0.f};
+  float col[4] = {0.f, 0.f, 0.f, 0.f}, col_sq[4] = {0.f, 0.f, 0.f, 0.f};
+  const int counted_from = rule_first_counted_row(c.rule, c.window, a.I, c.g);   // rules that look at the last queries only
   const int first_row = (j0 > c.n_old) ? (j0 - c.n_old) * c.g : 0;  // earlier rows cannot see this tile
   for (int row0 = (first_row / kTile) * kTile; row0 < R; row0 += kTile) {
     __syncthreads();
     load_tile<T, D>(sQ, tid, [&](int r) { return query_row_ptr<T, D>(c, a, smp, kh, row0 + r); });
-    // rule 2 (current query): only the rows of the block's last input contribute
     if (tid < kTile)
-      sLse[tid] = (row0 + tid < R && (c.rule != 2 || row0 + tid >= R - c.g)) ? a.lse[(size_t)unit * R + row0 + tid] : INFINITY;
+      sLse[tid] = (row0 + tid < R && row0 + tid >= counted_from) ? a.lse[(size_t)unit * R + row0 + tid] : INFINITY;
     __syncthreads();
     float acc[4][4];
     dot_tile<D>(sQ, sK, ty, tx, acc);
 #pragma unroll
     for (int y = 0; y < 4; ++y) {
       const int j = j0 + tx + 16 * y;
-      float part = 0.f;
+      float part = 0.f, part_sq = 0.f;
 #pragma unroll
       for (int x = 0; x < 4; ++x) {
         const int r = ty + 16 * x, row = row0 + r;
         const bool vis = (row < R) && (j < c.n_old + row / c.g + 1);
-        part += vis ? expf(acc[x][y] * a.scale - sLse[r]) : 0.f;
+        const float w = vis ? expf(acc[x][y] * a.scale - sLse[r]) : 0.f;
+        part += w;
+        part_sq = fmaf(w, w, part_sq);
       }
       col[y] += part;
+      col_sq[y] += part_sq;
     }
   }
   __syncthreads();
@@ -235,10 +238,24 @@ __global__ void __launch_bounds__(kThreads) score_simt(CacheView c, BlockArgs a)
       if (pad > 0 && (j < c.n_old ? c.kv_ids[(size_t)unit * c.cap + j] : a.pos0 + (j - c.n_old)) < pad)
         tot = 0.f;                                  // a padding pair is masked for every query
       if (j < c.n_old) {
-        if (c.rule == 2) c.sum_weights[(size_t)unit * c.cap + j] = tot;   // nothing is carried over
+        if (rule_overwrites(c.rule)) c.sum_weights[(size_t)unit * c.cap + j] = tot;   // nothing is carried over
         else c.sum_weights[(size_t)unit * c.cap + j] += tot;
       }
       else a.new_sum[(size_t)unit * a.I + (j - c.n_old)] = tot;
+    }
+  }
+  if (c.sum_sq != nullptr) {    // rule 4: the same reduction over the squares
+    __syncthreads();
+#pragma unroll
+    for (int y = 0; y < 4; ++y) sRed[ty * kTile + tx + 16 * y] = col_sq[y];
+    __syncthreads();
+    if (tid < kTile && j0 + tid < n_c) {
+      const int j = j0 + tid;
+      float tot = 0.f;
+#pragma unroll
+      for (int t = 0; t < 16; ++t) tot += sRed[t * kTile + tid];
+      if (j < c.n_old) c.sum_sq[(size_t)unit * c.cap + j] += tot;
+      else a.new_sq[(size_t)unit * a.I + (j - c.n_old)] = tot;
     }
   }
 }

@@ -41,7 +41,11 @@ struct TcArgs {
   const int* left_pad;
   const int* kv_ids;
   int pos0;
-  int rule;          // 2: only the rows of the block's last input contribute to the column sums, which replace sum_weights
+  int rule;
+  int first_row;     // query rows below it add nothing to the column sums (rules that look at the last queries only)
+  int overwrite;     // 1: the column sums replace sum_weights instead of being added
+  float* sum_sq;     // rule 4: sums of squared weights (cached pairs / the block's pairs), else null
+  float* new_sq;
 };
 
 #include "attn_fwd_split.cuh"
@@ -70,7 +74,8 @@ struct ScoreSmem {
 enum { C_KFULL = 0, C_QFULL = 1, C_QEMPTY = C_QFULL + kQStages, C_SFULL = C_QEMPTY + kQStages,
        C_SFREE = C_SFULL + kScoreWG, C_COUNT = C_SFREE + kScoreWG };
 
-template <int D>
+// SQ: the sums of squared weights are taken as well (rule 4; an instance of its own, so that the others carry none of it)
+template <int D, bool SQ>
 __global__ void __launch_bounds__(kScoreThreads, 2)
 score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   using L = ScoreSmem<D>;
@@ -160,13 +165,13 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
     const int key = quad * 32 + lane;              // key inside the tile == TMEM lane
     const uint32_t ts = tmem + wg * 128 + ((uint32_t)(quad * 32) << 16);
     const float* lse_w = sLse + wg * 128;
-    float acc = 0.f;
+    float acc = 0.f, acc_sq = 0.f;
     for (int t = wg; t < T; t += kScoreWG) {
       const int qrow0 = (qt0 + t) * kTileM;
       // this tile's log2-sum-exp values; +inf for rows past the block's end (weight 0)
       {
         const int rr = qrow0 + key;
-        sLse[wg * 128 + key] = (rr < R && (a.rule != 2 || rr >= R - a.g)) ? a.lse2[(size_t)unit * R + rr] : INFINITY;
+        sLse[wg * 128 + key] = (rr < R && rr >= a.first_row) ? a.lse2[(size_t)unit * R + rr] : INFINITY;
       }
       named_bar_sync(1 + wg, 128);
       mbar_wait(&bars[C_SFULL + wg], (t / kScoreWG) & 1, abort_flag, a.status);
@@ -174,7 +179,7 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
       // first query row of the tile that may see this key (causal mask inside the block)
       const int first_vis = is_old ? 0 : max(0, (c0 + key) * a.g - qrow0);
       const bool nomask = __all_sync(0xffffffffu, first_vis == 0);
-      float p0 = 0.f, p1 = 0.f;
+      float p0 = 0.f, p1 = 0.f, q0 = 0.f, q1 = 0.f;
       uint32_t cur[32], nxt[32];
       tmem_ld32(ts, cur);
       tmem_wait_ld();
@@ -192,6 +197,7 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
             e1 = col + 1 >= first_vis ? e1 : 0.f;
           }
           add2(p0, p1, e0, e1);
+          if (SQ) { q0 = fmaf(e0, e0, q0); q1 = fmaf(e1, e1, q1); }
         }
         if (cc < 3) {
           tmem_wait_ld();
@@ -200,16 +206,22 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
         }
       }
       acc += p0 + p1;
+      if (SQ) acc_sq += q0 + q1;
       tc_fence_before();
       mbar_arrive(&bars[C_SFREE + wg]);
       named_bar_sync(1 + wg, 128);                 // everyone is done with this tile's sLse before it is rewritten
     }
     sPart[wg * 128 + key] = acc;
+    if (SQ) sLse[wg * 128 + key] = acc_sq;         // (the last tile's values are no longer needed: barrier above)
     named_bar_sync(1 + kScoreWG, 128 * kScoreWG);
     if (wg == 0) {
-      float tot = 0.f;
+      float tot = 0.f, tot_sq = 0.f;
 #pragma unroll
       for (int w = 0; w < kScoreWG; ++w) tot += sPart[w * 128 + key];   // fixed order
+      if (SQ) {
+#pragma unroll
+        for (int w = 0; w < kScoreWG; ++w) tot_sq += sLse[w * 128 + key];
+      }
       const int j = is_old ? kt * kTileN + key : c0 + key;
       if (a.left_pad != nullptr) {                  // a padding pair is masked for every query
         const int pad = a.left_pad[smp];
@@ -218,11 +230,15 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
       }
       if (is_old) {
         if (j < a.n_old) {
-          if (a.rule == 2) a.sum_weights[(size_t)unit * a.cap + j] = tot;   // nothing is carried over
+          if (a.overwrite) a.sum_weights[(size_t)unit * a.cap + j] = tot;   // nothing is carried over
           else a.sum_weights[(size_t)unit * a.cap + j] += tot;
+          if (SQ) a.sum_sq[(size_t)unit * a.cap + j] += tot_sq;
         }
       }
-      else if (j < a.I) a.new_sum[(size_t)unit * a.I + j] = tot;
+      else if (j < a.I) {
+        a.new_sum[(size_t)unit * a.I + j] = tot;
+        if (SQ) a.new_sq[(size_t)unit * a.I + j] = tot_sq;
+      }
     }
   }
   tc_fence_before();
@@ -293,6 +309,9 @@ TcArgs make_args(const CacheView& c, const BlockArgs& a) {
   t.lse2 = a.lse; t.sum_weights = c.sum_weights; t.new_sum = a.new_sum;
   t.cap = c.cap; t.status = c.status;
   t.left_pad = c.left_pad; t.kv_ids = c.kv_ids; t.pos0 = a.pos0; t.rule = c.rule;
+  t.first_row = rule_first_counted_row(c.rule, c.window, a.I, c.g);
+  t.overwrite = rule_overwrites(c.rule) ? 1 : 0;
+  t.sum_sq = c.sum_sq; t.new_sq = a.new_sq;
   return t;
 }
 
@@ -320,7 +339,7 @@ thread_local bool g_scores_done = false;
 // under a rule that accumulates every row's weights: forward pass and column sums in one kernel (attn_onepass.cuh).
 bool onepass_applies(const CacheView& c, const BlockArgs& a) {
   const int t_old = (c.n_old + kTileN - 1) / kTileN, t_new = (a.I + kTileN - 1) / kTileN;
-  return c.left_pad == nullptr && c.rule != 2 && a.I * c.g <= kTileM && t_old + t_new <= 4;
+  return c.left_pad == nullptr && c.rule <= 1 && a.I * c.g <= kTileM && t_old + t_new <= 4;
 }
 
 template <int D>
@@ -341,16 +360,20 @@ cudaError_t launch_fwd_t(const CacheView& c, const BlockArgs& a, cudaStream_t st
   return c.left_pad != nullptr ? launch_fwd_split<D, true>(c, a, st) : launch_fwd_split<D, false>(c, a, st);
 }
 
-template <int D>
-cudaError_t launch_score_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+template <int D, bool SQ>
+cudaError_t launch_score_sq(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
   static SmemConfigured configured;
-  if (cudaError_t e = configured.ensure(score_tc<D>, (size_t)(ScoreSmem<D>::kTotal)); e != cudaSuccess) return e;
+  if (cudaError_t e = configured.ensure(score_tc<D, SQ>, (size_t)(ScoreSmem<D>::kTotal)); e != cudaSuccess) return e;
   const int t_old = (c.n_old + kTileN - 1) / kTileN, t_new = (a.I + kTileN - 1) / kTileN;
   dim3 grid(t_old + t_new, c.nsamples * c.Hkv);
   ProfileScope prof(kScore, st);
-  score_tc<D><<<grid, kScoreThreads, ScoreSmem<D>::kTotal, st>>>(g_maps, make_args(c, a));
+  score_tc<D, SQ><<<grid, kScoreThreads, ScoreSmem<D>::kTotal, st>>>(g_maps, make_args(c, a));
   count_launch();
   return cudaGetLastError();
+}
+template <int D>
+cudaError_t launch_score_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+  return c.sum_sq != nullptr ? launch_score_sq<D, true>(c, a, st) : launch_score_sq<D, false>(c, a, st);
 }
 
 // Self-test of the bounded wait: one thread waits on a barrier that nothing ever arrives on.  The wait gives up

@@ -20,9 +20,21 @@ struct CacheView {
   int32_t* status;     // device status word
   const int32_t* left_pad;  // [nsamples] padding positions at the start of each sample of the range, or null
   unsigned long long* moved;  // [16] counters of rows moved by compactions (unit & 15), or null when not counting
-  int32_t rule;             // 0 average attention (Sec. 3.2), 1 sum + window of recent pairs, 2 current query (Sec. 2)
+  int32_t rule;             // 0 average attention (Sec. 3.2); Sec. 2: 1 sum + window of recent pairs, 2 current query,
+                            // 3 last-window sums, pooled, recent window kept, 4 average + standard deviation
   int32_t fill;             // 1: unordered cache -- pairs that stay never move, new pairs fill the freed rows
+  float* sum_sq;            // [units][cap] sums of squared attention weights (rule 4), else null
+  int32_t window, pool;     // rule 3: queries observed / recent pairs kept; width of the max-pooling (odd)
+  int32_t std_permille;     // rule 4: share of the kept pairs chosen by standard deviation, in 1/1000
 };
+
+// Rules that rank by recent queries only (Sec. 2): sum_weights is overwritten by every pass, and only the rows of the
+// pass's last inputs count -- its last input (rule 2) or its last min(window, I) inputs (rule 3).
+__host__ __device__ inline bool rule_overwrites(int rule) { return rule == 2 || rule == 3; }
+__host__ __device__ inline int rule_first_counted_row(int rule, int window, int I, int g) {
+  const int inputs = rule == 2 ? 1 : (rule == 3 ? (window < I ? window : I) : I);
+  return (I - inputs) * g;
+}
 
 // Left padding (Sec. 3): positions below the sample's count are padding.  A padding pair is masked for every
 // real query; a padding query produces a zero output row and no attention weights.
@@ -38,6 +50,7 @@ struct BlockArgs {
   void* out;        // [nsamples][I][Hq][d]
   float* lse;       // workspace: [units][I*g]  natural-log-sum-exp of every query row
   float* new_sum;   // workspace: [units][I]    column sums of the block's own pairs
+  float* new_sq;    // workspace: [units][I]    column sums of squares of the block's own pairs (rule 4), else null
   int32_t I;
   int32_t pos0;
   float scale;
@@ -47,6 +60,7 @@ struct EvictArgs {
   const void* blk_k;     // block K/V when the new pairs still live in the caller's buffers, else null
   const void* blk_v;
   const float* new_sum;  // [units][I] when I > 0
+  const float* new_sq = nullptr;  // [units][I] when I > 0 under rule 4
   int32_t I;             // candidates = n_old + I
   int32_t pos0;
   int32_t curr_id;       // last processed position

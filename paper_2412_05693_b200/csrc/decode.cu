@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
   T* kslab = reinterpret_cast<T*>(c.k_slab) + base * D;
   T* vslab = reinterpret_cast<T*>(c.v_slab) + base * D;
   // (an unordered cache takes the general path for every cut: there the new pair fills the freed row)
-  const bool evict_one = (a.target == n1 - 1) && !c.fill;
+  const bool evict_one = (a.target == n1 - 1) && !c.fill && c.rule < 3;   // rules 3, 4 rank by more than one value per pair
   const bool evict_general = (a.target >= 0 && a.target < n1 && !evict_one);
   // left-padded sample: padding pairs are masked and leave first; a query at a padding position (not a real
   // decode step) gets a zero output and no weights
@@ -197,8 +197,14 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
       s.p[h * n1p + j] = p;
       add += p;
     }
-    // rule 2 (current query) keeps this step's weights only
-    const float sw = ((j < c.n_old && c.rule != 2) ? c.sum_weights[base + j] : 0.f) + add;
+    // rules 2 and 3 (recent queries only) keep this step's weights only
+    const float sw = ((j < c.n_old && !rule_overwrites(c.rule)) ? c.sum_weights[base + j] : 0.f) + add;
+    if (c.sum_sq != nullptr) {                                       // rule 4: sum of squared weights as well
+      float add_sq = 0.f;
+#pragma unroll
+      for (int h = 0; h < G; ++h) add_sq = fmaf(s.p[h * n1p + j], s.p[h * n1p + j], add_sq);
+      c.sum_sq[base + j] = (j < c.n_old ? c.sum_sq[base + j] : 0.f) + add_sq;
+    }
     s.score[j] = sw;
     if (evict_one) {
       float ave;   // ranking value: average attention (Sec. 3.2), or the raw weights with / without a recent window

@@ -132,7 +132,8 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
   T* vslab = reinterpret_cast<T*>(c.v_slab) + base * D;
   // (an unordered cache under the rule with a window of recent pairs takes the general path for every cut: the
   // window is a select on kv_ids there)
-  const bool evict_one = (a.target == n1 - 1) && (PLAIN || !(c.fill && c.rule == 1));
+  // (so do the rules whose ranking is more than one value per pair: pooled window sums, deviation-protected averages)
+  const bool evict_one = (a.target == n1 - 1) && (PLAIN || !((c.fill && c.rule == 1) || c.rule >= 3));
   const bool evict_general = (a.target >= 0 && a.target < n1 && !evict_one);
 
   // Programmatic dependent launch: this grid may have been started while its predecessor in the stream was still
@@ -366,7 +367,13 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
     } else if (j < c.n_old) {
       old_sw = c.sum_weights[base + j];
     }
-    const float sw = (rule == 2 ? 0.f : old_sw) + add;   // rule 2 (current query) keeps this step's weights only
+    const float sw = (rule_overwrites(rule) ? 0.f : old_sw) + add;   // rules 2, 3 keep this step's weights only
+    if (!PLAIN && c.sum_sq != nullptr) {                             // rule 4: sum of squared weights as well
+      float add_sq = 0.f;
+#pragma unroll
+      for (int h = 0; h < G; ++h) add_sq = fmaf(s.p[h * n1t + j], s.p[h * n1t + j], add_sq);
+      c.sum_sq[base + j] = (j < c.n_old ? c.sum_sq[base + j] : 0.f) + add_sq;
+    }
     s.score[j] = sw;
     if (evict_one) {
       float ave;   // ranking value: average attention (Sec. 3.2), or the raw weights with / without a recent window

@@ -81,11 +81,22 @@ __device__ inline void evict_body_impl(const CacheView& c, int unit, int smp, in
   const float gf = (float)c.g;
   const int pad = sample_left_pad(c, smp);
   int id_win = 0x7fffffff;   // unordered cache, rule 1: pairs at positions >= id_win form the window of recent pairs
+  // rule 3 (Sec. 2, SnapKV): the min(window, target) most recent candidates always stay; every other score is replaced
+  // by the maximum over the `pool` neighbours centred on it, the window left out
+  const int pool_body = n_c - min(c.window, target), pool_half = c.pool / 2;
   auto ave_bits = [&](int j) -> uint32_t {
     const float cnt = (float)(e.curr_id + 1 - s.id[j]);
     uint32_t b;   // ranking value >= 0: the bit pattern orders like the value
-    if (c.rule == 0) b = __float_as_uint(s.score[j] / (gf * cnt));       // average attention (Sec. 3.2)
+    if (c.rule == 0 || c.rule == 4) b = __float_as_uint(s.score[j] / (gf * cnt));   // average attention (Sec. 3.2)
     else if (c.rule == 1 && (FILL ? s.id[j] >= id_win : j >= n_c - target / 2)) b = 0x7f800000u;   // recent window: always kept
+    else if (c.rule == 3) {
+      if (j >= pool_body) b = 0x7f800000u;
+      else {
+        float m = s.score[j];
+        for (int x = max(0, j - pool_half); x < min(pool_body, j + pool_half + 1); ++x) m = fmaxf(m, s.score[x]);
+        b = __float_as_uint(m);
+      }
+    }
     else b = __float_as_uint(s.score[j]);                                // raw (sum of / current) weights
     if (pad == 0) return b;
     return s.id[j] < pad ? 0u : max(b, 1u);   // padding pairs rank below every real pair (left-padded samples)
@@ -220,7 +231,36 @@ __device__ inline void evict_body_impl(const CacheView& c, int unit, int smp, in
     // ---- radix select: bit pattern `thr` of the target-th largest ave, and how many equal to it to keep
     uint32_t thr;
     int need_eq;
-    for (int j = tid; j < n_c; j += NT) s.bits[j] = ave_bits(j);   // one division per candidate, not one per pass
+    const int n_std = c.rule == 4 ? (int)(((long long)target * c.std_permille) / 1000) : 0;
+    if (n_std > 0) {
+      // rule 4 (Sec. 2 / Sec. 3.2, RoCo): the n_std candidates whose weights have the largest standard deviation,
+      // sqrt(E[w^2] - E[w]^2) over the g * (curr_id + 1 - kv_ids) weights received, stay whatever their average
+      // (ties: lower position first); they enter the ranking below as +inf, the others with their average
+      for (int j = tid; j < n_c; j += NT) {
+        const float cnt = gf * (float)(e.curr_id + 1 - s.id[j]);
+        const float sq = j < n_old ? c.sum_sq[base + j] : e.new_sq[(size_t)unit * e.I + (j - n_old)];
+        const float mean = s.score[j] / cnt;
+        s.bits[j] = __float_as_uint(sqrtf(fmaxf(sq / cnt - mean * mean, 0.f)));
+      }
+      __syncthreads();
+      uint32_t thr_s;
+      int need_s;
+      radix_kth_largest([&](int j, uint32_t& key) { key = s.bits[j]; return true; }, n_std, thr_s, need_s);
+      const int chunk = (n_c + NT - 1) / NT;
+      const int jb = min(tid * chunk, n_c), je = min(jb + chunk, n_c);
+      int eq = 0;
+      for (int j = jb; j < je; ++j) eq += (s.bits[j] == thr_s);
+      int unused, eq_before;
+      block_exclusive_scan2<NT>(0, eq, s.wsum, unused, eq_before);
+      for (int j = jb; j < je; ++j) {       // every thread rewrites its own chunk only
+        const uint32_t b = s.bits[j];
+        const bool prot = b > thr_s || (b == thr_s && eq_before < need_s);
+        eq_before += (b == thr_s);
+        s.bits[j] = prot ? 0x7f800000u : ave_bits(j);
+      }
+    } else {
+      for (int j = tid; j < n_c; j += NT) s.bits[j] = ave_bits(j);   // one division per candidate, not one per pass
+    }
     __syncthreads();
     radix_kth_largest([&](int j, uint32_t& key) { key = s.bits[j]; return true; }, target, thr, need_eq);
     if constexpr (FILL) {
@@ -281,6 +321,14 @@ __device__ inline void evict_body_impl(const CacheView& c, int unit, int smp, in
     const int j = s.src[r];
     c.sum_weights[base + r] = s.score[j];
     c.kv_ids[base + r] = s.id[j];
+  }
+  if (c.sum_sq != nullptr) {
+    // rule 4: the sums of squares take the same places; they pass through shared memory (the ranking values are no
+    // longer needed), so that every load has completed before the first store
+    for (int j = tid; j < n_c; j += NT)
+      s.bits[j] = __float_as_uint(j < n_old ? c.sum_sq[base + j] : e.new_sq[(size_t)unit * e.I + (j - n_old)]);
+    __syncthreads();
+    for (int r = first_moved + tid; r < target; r += NT) c.sum_sq[base + r] = __uint_as_float(s.bits[s.src[r]]);
   }
 
   // ---- rows: ascending chunks, every source row index >= its destination, loads of a chunk complete

@@ -169,10 +169,10 @@ def schedule(wl: Workload):
 
 
 def config_for(wl: Workload, device: int = 0, growth: int | None = None, batch: int | None = None,
-               max_call_samples: int = 0, rule: str = "average", compaction: str = "stable"):
+               max_call_samples: int = 0, rule: str = "average", compaction: str = "stable", **rule_params):
     """The library configuration of a workload in the build's cadence (cap = kv_max + growth)."""
     from .binding import Config
     return Config(batch=wl.b if batch is None else batch, n_q_heads=wl.Hq, n_kv_heads=wl.Hkv, head_dim=wl.d,
                   kv_max=wl.K, block_max=wl.B, growth=max(1, wl.p_dec) if growth is None else growth,
                   dtype=wl.dtype, n_layers=wl.L, device=device, max_call_samples=max_call_samples, rule=rule,
-                  compaction=compaction)
+                  compaction=compaction, **rule_params)   # window / pool / std_share of the rules that take them

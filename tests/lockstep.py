@@ -23,8 +23,8 @@ OUT_TOL = {"bf16": 2e-2, "f32": 1e-4}
 
 
 def make_config(wl: Workload, device: int = 0, growth: int | None = None, batch: int | None = None,
-                max_call_samples: int = 0, rule: str = "average", compaction: str = "stable") -> Config:
-    return config_for(wl, device, growth, batch, max_call_samples, rule, compaction)
+                max_call_samples: int = 0, rule: str = "average", compaction: str = "stable", **rule_params) -> Config:
+    return config_for(wl, device, growth, batch, max_call_samples, rule, compaction, **rule_params)
 
 
 def _np(t):
@@ -68,10 +68,55 @@ def check_kept(unit: UnitCache, gpu_ids: np.ndarray, target: int, stats: dict, w
     stats["evictions"] += 1
 
 
+STD_BAND = 2e-3   # relative band around the deviation cut: sqrt(E[w^2] - E[w]^2) in fp32 loses digits to cancellation
+
+
+def check_kept_average_std(unit: UnitCache, gpu_ids: np.ndarray, target: int, stats: dict, where: str):
+    """The rule with pairs protected by the standard deviation of their weights (Sec. 2, RoCo): two cuts, so the
+    band check has two stages.  A pair whose deviation is clearly above the deviation cut must be kept; a pair near
+    that cut may have been chosen by either side; every other pair is judged by its average against the averages
+    next to the average cut (one rank of slack, since a different choice at the first cut shifts the second by one)."""
+    if target == 0:
+        assert len(gpu_ids) == 0
+        unit.evict(0)
+        stats["evictions"] += 1
+        return
+    cand = unit.kv_ids
+    gpu = np.asarray(gpu_ids, dtype=np.int64)
+    assert gpu.shape[0] == target and np.all(np.diff(gpu) > 0) and np.isin(gpu, cand).all(), f"{where}: bad kept set"
+    ave = unit.ave_weights()
+    cnt = unit.g * (unit.last_pos + 1 - cand)
+    std = np.sqrt(np.maximum(unit.sum_sq / cnt - ave * ave, 0.0))
+    n_std = int(np.floor(unit.std_share * target + 1e-9))
+    kept = np.isin(cand, gpu)
+    near = np.zeros(len(cand), dtype=bool)
+    sure = np.zeros(len(cand), dtype=bool)
+    if n_std > 0:
+        cut_s = np.sort(std)[::-1][n_std - 1]
+        sure = std > cut_s * (1 + STD_BAND)
+        near = (std >= cut_s * (1 - STD_BAND)) & ~sure
+        assert not np.any(sure & ~kept), f"{where}: dropped a pair whose deviation is clearly above the cut"
+    score = unit.ranking_scores(target)                       # the oracle's own choice: protected pairs at +inf
+    order = np.lexsort((cand, -score))
+    rest = order[n_std:]                                      # by average, best first
+    k = target - n_std                                        # pairs chosen by average
+    if 0 < k < len(rest):
+        hi = ave[rest[max(k - 2, 0)]]                         # one rank better than the last pair chosen by average
+        lo = ave[rest[min(k + 1, len(rest) - 1)]]             # one rank worse than the first pair not chosen
+        judged = ~sure & ~near
+        assert not np.any(judged & ~kept & (ave > hi * (1 + BAND))), f"{where}: dropped a pair clearly above the average cut"
+        assert not np.any(judged & kept & (ave < lo * (1 - BAND))), f"{where}: kept a pair clearly below the average cut"
+    own = cand[np.sort(order[:target])]
+    if not np.array_equal(own, gpu):
+        stats["adoptions"] += 1
+    unit.evict(target, kept_ids=gpu)
+    stats["evictions"] += 1
+
+
 def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=None, check_rows_every: int = 8,
                  growth: int | None = None, sum_rtol: float | None = None, pads=None, rule: str = "average",
                  compaction: str = "stable", micro: int | None = None, micro_dec: int | None = None, arena=None,
-                 cache=None):
+                 cache=None, rule_params: dict | None = None):
     """Run `calls` (default: the workload's spec schedule) on the GPU for the whole batch and on the
     oracle for `units` = [(sample, kv_head), ...].  Returns a dict of statistics; raises on any mismatch.
 
@@ -84,12 +129,14 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
     own_cache = cache is None
     if own_cache:
         mc = 0 if micro is None else max(micro, micro_dec or micro)
-        cfg = make_config(wl, device, growth, rule=rule, compaction=compaction, max_call_samples=min(mc, wl.b))
+        cfg = make_config(wl, device, growth, rule=rule, compaction=compaction, max_call_samples=min(mc, wl.b),
+                          **(rule_params or {}))
         cache = BatchMaxCache(cfg, arena=arena)
     if pads is not None:                            # left-padded samples: pads[sample] padding positions
         cache.set_left_pad(pads)
     g = wl.g
-    oracles = {u: UnitCache(wl.d, g, left_pad=0 if pads is None else pads[u[0]], rule=rule) for u in units}
+    oracles = {u: UnitCache(wl.d, g, left_pad=0 if pads is None else pads[u[0]], rule=rule, **(rule_params or {}))
+               for u in units}
     stats = {"adoptions": 0, "evictions": 0, "max_out_err": 0.0, "max_sum_rel": 0.0, "calls": 0, "tc_calls": 0,
              "onepass_calls": 0}
     tol = OUT_TOL[wl.dtype]
@@ -149,7 +196,10 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
                 if want_rows:
                     kr, vr = kr[torch.from_numpy(order)], vr[torch.from_numpy(order)]
             if kind != "recent" and evict_to >= 0 and len(unit) > evict_to:
-                check_kept(unit, ids, evict_to, stats, where)
+                if rule == "average_std":
+                    check_kept_average_std(unit, ids, evict_to, stats, where)
+                else:
+                    check_kept(unit, ids, evict_to, stats, where)
             assert np.array_equal(ids, unit.kv_ids), f"{where}: kv_ids differ from the oracle's"
             n_gpu, cur = cache.length(layer, smp)
             assert n_gpu == len(unit) and cur == unit.last_pos, f"{where}: host mirror n/curr_id wrong"
@@ -158,6 +208,10 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
                 if len(unit) else 0.0              # (an eviction call on a still-empty cache is legal)
             stats["max_sum_rel"] = max(stats["max_sum_rel"], rel)
             assert rel <= sum_rtol, f"{where}: sum_weights relative error {rel:.3e} > {sum_rtol}"
+            if rule == "average_std" and len(unit):
+                sq = cache.export_sum_sq(layer, smp, kh).numpy().astype(np.float64)
+                rel = float(np.max(np.abs(sq - unit.sum_sq) / np.maximum(np.abs(unit.sum_sq), 1e-4)))
+                assert rel <= sum_rtol, f"{where}: sums of squared weights off by {rel:.3e} > {sum_rtol}"
             if want_rows:
                 assert np.array_equal(_np(kr), unit.k), f"{where}: cached K rows are not the oracle's rows"
                 assert np.array_equal(_np(vr), unit.v), f"{where}: cached V rows are not the oracle's rows"

@@ -137,6 +137,25 @@ def test_random_cadences_rules_and_padding(seed):
         run_lockstep(wl, all_units(wl)[:3], pads=pads, rule=rule, check_rows_every=3)
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_random_cadences_of_the_pooled_window_and_deviation_rules(seed):
+    # the two rules with parameters of their own (Sec. 2: SnapKV, RoCo) under any cadence of the four calls
+    rng = np.random.default_rng(5200 + seed)
+    g, hkv, d = int(rng.choice([1, 2, 4])), int(rng.integers(1, 4)), int(rng.choice([64, 128]))
+    wl = Workload(f"cad2_{seed}", b=int(rng.integers(1, 4)), Hq=g * hkv, Hkv=hkv, d=d, dtype=str(rng.choice(["bf16", "f32"])),
+                  s=int(rng.integers(50, 700)), B=int(rng.integers(1, 250)), K=int(rng.integers(1, 300)),
+                  steps=int(rng.integers(0, 12)), seed=5200 + seed, heavy_count=3, p_dec=int(rng.choice([1, 3])))
+    calls, growth = random_cadence(wl, rng)
+    if seed % 2 == 0:
+        params = dict(window=int(rng.integers(1, 80)), pool=int(rng.choice([1, 3, 5, 9])))
+        run_lockstep(wl, all_units(wl)[:3], calls=calls, growth=growth, rule="window_pooled", rule_params=params,
+                     check_rows_every=3)
+    else:
+        params = dict(std_share=float(rng.choice([0.1, 0.333, 0.5, 0.9])))
+        run_lockstep(wl, all_units(wl)[:3], calls=calls, growth=growth, rule="average_std", rule_params=params,
+                     check_rows_every=3)
+
+
 # ------------------------------------------------------------------ shapes, tails and degenerate cases
 @pytest.mark.parametrize("wl", [
     tiny("ragged_f32"),                                               # I = 48, tail of 8, g = 2
@@ -376,6 +395,56 @@ def test_alternative_eviction_rules_lockstep(rule, dtype, d, Hq, Hkv):
     wl = tiny("rules", s=400, B=128, K=96, steps=12, dtype=dtype, d=d, Hq=Hq, Hkv=Hkv)
     st = run_lockstep(wl, all_units(wl), rule=rule, check_rows_every=2)
     assert st["evictions"] >= 2 * Hkv * (3 + 12)
+
+
+@pytest.mark.parametrize("window,pool", [(1, 1), (8, 3), (16, 7), (64, 5)])
+@pytest.mark.parametrize("dtype,d,Hq,Hkv,B,K", [("bf16", 128, 8, 2, 48, 40), ("f32", 64, 4, 4, 20, 33), ("bf16", 128, 4, 4, 160, 150)])
+def test_window_pooled_rule_lockstep(window, pool, dtype, d, Hq, Hkv, B, K):
+    # Sec. 2, SnapKV: sums over the last `window` queries of the pass, max-pooled over neighbours, recent window kept
+    wl = tiny(f"snap_{dtype}_w{window}_p{pool}", dtype=dtype, d=d, Hq=Hq, Hkv=Hkv, s=3 * B + 7, B=B, K=K, steps=5)
+    st = run_lockstep(wl, all_units(wl), rule="window_pooled", rule_params=dict(window=window, pool=pool),
+                      check_rows_every=2)
+    assert st["evictions"] > 0
+
+
+def test_window_pooled_rule_one_compression_after_the_prompt():
+    # the rule's own cadence (Sec. 2): nothing leaves during prefilling, one compression after the prompt
+    wl = tiny("snap_once", dtype="bf16", d=128, Hq=8, Hkv=2, s=300, B=64, K=96, steps=4)
+    calls = [("prefill", p, min(wl.B, wl.s - p), -1) for p in range(0, wl.s, wl.B)] + [("evict", 0, 0, wl.K)]
+    calls += [("decode", wl.s + t, 1, -1) for t in range(wl.steps)]
+    st = run_lockstep(wl, all_units(wl), calls=calls, growth=wl.s + wl.steps - wl.K, rule="window_pooled",
+                      rule_params=dict(window=32, pool=7), check_rows_every=2)
+    assert st["evictions"] == len(all_units(wl))
+
+
+def test_window_pooled_rule_with_left_padding():
+    wl = tiny("snap_pad", dtype="bf16", d=128, Hq=8, Hkv=2, s=200, B=40, K=48, steps=6)
+    run_lockstep(wl, all_units(wl), pads=[0, 57], rule="window_pooled", rule_params=dict(window=8, pool=3),
+                 check_rows_every=2)
+
+
+@pytest.mark.parametrize("share", [0.0, 0.25, 0.5, 1.0])
+@pytest.mark.parametrize("dtype,d,Hq,Hkv,B,K,p_dec", [("bf16", 128, 8, 2, 48, 40, 1), ("f32", 64, 4, 4, 20, 33, 1),
+                                                       ("bf16", 128, 4, 4, 160, 150, 4)])
+def test_average_std_rule_lockstep(share, dtype, d, Hq, Hkv, B, K, p_dec):
+    # Sec. 2 / Sec. 3.2 last paragraph, RoCo: part of the kept pairs by the standard deviation of their weights
+    wl = tiny(f"roco_{dtype}_{share}", dtype=dtype, d=d, Hq=Hq, Hkv=Hkv, s=3 * B + 7, B=B, K=K, steps=9, p_dec=p_dec)
+    st = run_lockstep(wl, all_units(wl), rule="average_std", rule_params=dict(std_share=share), check_rows_every=2)
+    assert st["evictions"] > 0
+
+
+def test_rules_that_need_ordered_rows_refuse_unordered_caches_and_padding():
+    wl = tiny("refuse", dtype="bf16", d=128)
+    for rule in ("window_pooled", "average_std"):
+        with pytest.raises(bm.BMError):
+            bm.arena_bytes(make_config(wl, rule=rule, compaction="fill"))
+    cache = bm.BatchMaxCache(make_config(wl, rule="average_std"))
+    with pytest.raises(bm.BMError):
+        cache.set_left_pad([0, 3])
+    # the memory model charges the second accumulator: 4 more bytes per row
+    a = bm.cache_bytes_per_sample(make_config(wl, rule="average_std"))
+    b = bm.cache_bytes_per_sample(make_config(wl, rule="average"))
+    assert a - b == 4 * wl.Hkv * (wl.K + 1)
 
 
 def test_alternative_rule_with_left_padding():
