@@ -230,32 +230,38 @@ __global__ void __launch_bounds__(320, 2) attn_fwd_split(const __grid_constant__
       float ps0 = 0.f, ps1 = 0.f;
       const float neg_m = -m_used;
       // second read of the logits, 32 columns at a time (keeps the register count inside two CTAs per SM); the
-      // bf16 pairs of each chunk go over this thread's own logits: columns [64 half, 64 half + 32)
+      // bf16 pairs of each chunk go over this thread's own logits: columns [64 half, 64 half + 32).  The loop exists
+      // twice, with and without masks: as one loop with a test inside, the compiler evaluated the masks of every
+      // tile (two more instructions per exponential on the fully visible tiles, which are most).
+      auto exp_chunks = [&](auto masked) {
 #pragma unroll
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t sv[32], pk[16];
-        tmem_ld32(tm_s + lane_addr + c_lo + 32 * ch, sv);
-        tmem_wait_ld();
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t sv[32], pk[16];
+          tmem_ld32(tm_s + lane_addr + c_lo + 32 * ch, sv);
+          tmem_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-          float x0, x1;
-          fma2(x0, x1, __uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1]), a.scale_log2, neg_m);
-          float p0 = ex2(x0), p1 = ex2(x1);
-          if (!full) {
-            const int c0 = c_lo + 32 * ch + 2 * e;
-            p0 = (c0 < nvis && c0 >= nlo && !((pm >> (32 * ch + 2 * e)) & 1)) ? p0 : 0.f;
-            p1 = (c0 + 1 < nvis && c0 + 1 >= nlo && !((pm >> (32 * ch + 2 * e + 1)) & 1)) ? p1 : 0.f;
+          for (int e = 0; e < 16; ++e) {
+            float x0, x1;
+            fma2(x0, x1, __uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1]), a.scale_log2, neg_m);
+            float p0 = ex2(x0), p1 = ex2(x1);
+            if (decltype(masked)::value) {
+              const int c0 = c_lo + 32 * ch + 2 * e;
+              p0 = (c0 < nvis && c0 >= nlo && !((pm >> (32 * ch + 2 * e)) & 1)) ? p0 : 0.f;
+              p1 = (c0 + 1 < nvis && c0 + 1 >= nlo && !((pm >> (32 * ch + 2 * e + 1)) & 1)) ? p1 : 0.f;
+            }
+            add2(ps0, ps1, p0, p1);
+            pk[e] = pack_bf16(p0, p1);
           }
-          add2(ps0, ps1, p0, p1);
-          pk[e] = pack_bf16(p0, p1);
+          tmem_st16(tm_s + lane_addr + c_lo + 16 * ch, pk);
+          if (ch == 0) {                              // the first half may enter P.V now
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&bars[B_PHALF]);
+          }
         }
-        tmem_st16(tm_s + lane_addr + c_lo + 16 * ch, pk);
-        if (ch == 0) {                              // the first half may enter P.V now
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(&bars[B_PHALF]);
-        }
-      }
+      };
+      if (full) exp_chunks(std::false_type{});
+      else exp_chunks(std::true_type{});
       l += ps0 + ps1;
       tmem_wait_st();
       tc_fence_before();

@@ -7,6 +7,8 @@
 //                 in a fixed order (deterministic, no atomics).
 // Query rows of a unit are ordered r = i * g + h (input i, head h of the group), so a tile of 128 rows shares
 // its K/V tiles among the g heads of the group.
+#include <type_traits>
+
 #include "tc_common.cuh"
 #include "common.cuh"
 
@@ -180,31 +182,37 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
       const int first_vis = is_old ? 0 : max(0, (c0 + key) * a.g - qrow0);
       const bool nomask = __all_sync(0xffffffffu, first_vis == 0);
       float p0 = 0.f, p1 = 0.f, q0 = 0.f, q1 = 0.f;
-      uint32_t cur[32], nxt[32];
-      tmem_ld32(ts, cur);
-      tmem_wait_ld();
+      // (the loop exists with and without the causal mask: as one loop with a test inside, the compiler evaluated
+      // the mask of every tile, two more instructions per exponential)
+      auto reduce_tile = [&](auto masked) {
+        uint32_t cur[32], nxt[32];
+        tmem_ld32(ts, cur);
+        tmem_wait_ld();
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        if (cc < 3) tmem_ld32(ts + (cc + 1) * 32, nxt);   // next chunk loads while this one is used
+        for (int cc = 0; cc < 4; ++cc) {
+          if (cc < 3) tmem_ld32(ts + (cc + 1) * 32, nxt);   // next chunk loads while this one is used
 #pragma unroll
-        for (int e = 0; e < 32; e += 2) {
-          const int col = cc * 32 + e;
-          float x0, x1;
-          fma2v(x0, x1, __uint_as_float(cur[e]), __uint_as_float(cur[e + 1]), a.scale_log2, -lse_w[col], -lse_w[col + 1]);
-          float e0 = ex2(x0), e1 = ex2(x1);
-          if (!nomask) {
-            e0 = col >= first_vis ? e0 : 0.f;
-            e1 = col + 1 >= first_vis ? e1 : 0.f;
+          for (int e = 0; e < 32; e += 2) {
+            const int col = cc * 32 + e;
+            float x0, x1;
+            fma2v(x0, x1, __uint_as_float(cur[e]), __uint_as_float(cur[e + 1]), a.scale_log2, -lse_w[col], -lse_w[col + 1]);
+            float e0 = ex2(x0), e1 = ex2(x1);
+            if (decltype(masked)::value) {
+              e0 = col >= first_vis ? e0 : 0.f;
+              e1 = col + 1 >= first_vis ? e1 : 0.f;
+            }
+            add2(p0, p1, e0, e1);
+            if (SQ) { q0 = fmaf(e0, e0, q0); q1 = fmaf(e1, e1, q1); }
           }
-          add2(p0, p1, e0, e1);
-          if (SQ) { q0 = fmaf(e0, e0, q0); q1 = fmaf(e1, e1, q1); }
-        }
-        if (cc < 3) {
-          tmem_wait_ld();
+          if (cc < 3) {
+            tmem_wait_ld();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) cur[e] = nxt[e];
+            for (int e = 0; e < 32; ++e) cur[e] = nxt[e];
+          }
         }
-      }
+      };
+      if (nomask) reduce_tile(std::false_type{});
+      else reduce_tile(std::true_type{});
       acc += p0 + p1;
       if (SQ) acc_sq += q0 + q1;
       tc_fence_before();

@@ -13,7 +13,8 @@ bool encode_slab_rows_map(CUtensorMap* m, const void* slab, int d, int rows, int
 namespace tc {
 
 constexpr int kErrTimeout = 6;            // BM_ERR_TIMEOUT
-constexpr int kWaitLimit = 1 << 21;       // try_wait polls before a wait gives up
+constexpr int kWaitLimit = 1 << 20;       // try_wait polls before a wait gives up (each may sleep up to kWaitSleepNs)
+constexpr uint32_t kWaitSleepNs = 1000;   // how long one poll may keep the thread suspended while the phase is open
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -32,16 +33,19 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* b) {
 // BM_ERR_TIMEOUT in the device status word and raises the CTA's abort flag; once the flag is up every
 // later wait returns at once, so the kernel runs to its normal end (TMEM release included) with
 // undefined results instead of hanging.
+// Each poll hands the thread to the hardware until the phase completes or the time hint runs out, so that a waiting
+// warp costs the SM's other warps next to no issue slots (polls that return at once made half of the forward
+// kernel's instructions).
 __device__ __forceinline__ void mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag, int* status,
                                           int limit = kWaitLimit) {
   if (*abort_flag) return;
   const uint32_t addr = smem_u32(b);
   for (int it = 0; it < limit; ++it) {
     uint32_t ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}\n"
-                 : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.b32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(addr), "r"(parity), "r"(kWaitSleepNs) : "memory");
     if (ok) return;
-    if ((it & 1023) == 1023 && *abort_flag) return;
+    if ((it & 255) == 255 && *abort_flag) return;
   }
   *abort_flag = 1;
   atomicExch(status, kErrTimeout);
