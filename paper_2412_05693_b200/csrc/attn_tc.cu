@@ -77,7 +77,7 @@ enum { C_KFULL = 0, C_QFULL = 1, C_QEMPTY = C_QFULL + kQStages, C_SFULL = C_QEMP
        C_SFREE = C_SFULL + kScoreWG, C_COUNT = C_SFREE + kScoreWG };
 
 // SQ: the sums of squared weights are taken as well (rule 4; an instance of its own, so that the others carry none of it)
-template <int D, bool SQ>
+template <int D, bool SQ, int EMU>
 __global__ void __launch_bounds__(kScoreThreads, 2)
 score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
   using L = ScoreSmem<D>;
@@ -196,7 +196,9 @@ score_tc(const __grid_constant__ TcMaps maps, const TcArgs a) {
             const int col = cc * 32 + e;
             float x0, x1;
             fma2v(x0, x1, __uint_as_float(cur[e]), __uint_as_float(cur[e + 1]), a.scale_log2, -lse_w[col], -lse_w[col + 1]);
-            float e0 = ex2(x0), e1 = ex2(x1);
+            float e0, e1;
+            if (EMU > 0 && ((e >> 1) % EMU) == EMU - 1) ex2_poly2(x0, x1, e0, e1);   // a share of the pairs off the special-function unit
+            else { e0 = ex2(x0); e1 = ex2(x1); }
             if (decltype(masked)::value) {
               e0 = col >= first_vis ? e0 : 0.f;
               e1 = col + 1 >= first_vis ? e1 : 0.f;
@@ -368,16 +370,25 @@ cudaError_t launch_fwd_t(const CacheView& c, const BlockArgs& a, cudaStream_t st
   return c.left_pad != nullptr ? launch_fwd_split<D, true>(c, a, st) : launch_fwd_split<D, false>(c, a, st);
 }
 
-template <int D, bool SQ>
-cudaError_t launch_score_sq(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+template <int D, bool SQ, int EMU>
+cudaError_t launch_score_emu(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
   static SmemConfigured configured;
-  if (cudaError_t e = configured.ensure(score_tc<D, SQ>, (size_t)(ScoreSmem<D>::kTotal)); e != cudaSuccess) return e;
+  if (cudaError_t e = configured.ensure(score_tc<D, SQ, EMU>, (size_t)(ScoreSmem<D>::kTotal)); e != cudaSuccess) return e;
   const int t_old = (c.n_old + kTileN - 1) / kTileN, t_new = (a.I + kTileN - 1) / kTileN;
   dim3 grid(t_old + t_new, c.nsamples * c.Hkv);
   ProfileScope prof(kScore, st);
-  score_tc<D, SQ><<<grid, kScoreThreads, ScoreSmem<D>::kTotal, st>>>(g_maps, make_args(c, a));
+  score_tc<D, SQ, EMU><<<grid, kScoreThreads, ScoreSmem<D>::kTotal, st>>>(g_maps, make_args(c, a));
   count_launch();
   return cudaGetLastError();
+}
+// Every fourth pair of exponentials of the score pass runs as a polynomial on the FMA and integer pipes
+// (ex2_poly2): the pass is bound by the special-function unit, and a quarter is where the instruction issue the
+// polynomial costs stops paying (measured at the cfg3 shape: -3.6 % at an eighth, -5.9 % at a quarter, -4.7 % at a
+// third, -0.6 % at a half).
+constexpr int kScoreEmu = 4;
+template <int D, bool SQ>
+cudaError_t launch_score_sq(const CacheView& c, const BlockArgs& a, cudaStream_t st) {
+  return launch_score_emu<D, SQ, kScoreEmu>(c, a, st);
 }
 template <int D>
 cudaError_t launch_score_t(const CacheView& c, const BlockArgs& a, cudaStream_t st) {

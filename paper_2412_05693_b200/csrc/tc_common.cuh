@@ -184,6 +184,35 @@ __device__ __forceinline__ void fma2v(float& d0, float& d1, float a0, float a1, 
       "fma.rn.f32x2 rd, ra, rb, rc;\nmov.b64 {%0, %1}, rd;\n}\n"
       : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b), "f"(c0), "f"(c1));
 }
+// (d0, d1) = (a0, a1) + (b0, b1) and (a0, a1) * (b0, b1) + (c0, c1), one packed instruction each
+__device__ __forceinline__ void add2g(float& d0, float& d1, float a0, float a1, float b0, float b1) {
+  asm("{\n.reg .b64 ra, rb, rd;\nmov.b64 ra, {%2, %3};\nmov.b64 rb, {%4, %5};\n"
+      "add.rn.f32x2 rd, ra, rb;\nmov.b64 {%0, %1}, rd;\n}\n"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+__device__ __forceinline__ void fma2g(float& d0, float& d1, float a0, float a1, float b0, float b1, float c0, float c1) {
+  asm("{\n.reg .b64 ra, rb, rc, rd;\nmov.b64 ra, {%2, %3};\nmov.b64 rb, {%4, %5};\nmov.b64 rc, {%6, %7};\n"
+      "fma.rn.f32x2 rd, ra, rb, rc;\nmov.b64 {%0, %1}, rd;\n}\n"
+      : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1), "f"(c0), "f"(c1));
+}
+// 2^x for a pair of x <= 0 on the FMA and integer pipes instead of the special-function unit: x = n + f with
+// n = round(x) (adding 1.5 * 2^23 leaves n in the low mantissa bits), 2^f by a degree-4 polynomial fitted on
+// [-1/2, 1/2] (relative error 2.7e-6), 2^n by adding n to the exponent field.  x below -126 gives 2^-126.
+__device__ __forceinline__ void ex2_poly2(float x0, float x1, float& r0, float& r1) {
+  constexpr float kMagic = 12582912.f;
+  x0 = fmaxf(x0, -126.f);
+  x1 = fmaxf(x1, -126.f);
+  float t0, t1, n0, n1, f0, f1, p0, p1;
+  add2g(t0, t1, x0, x1, kMagic, kMagic);
+  add2g(n0, n1, t0, t1, -kMagic, -kMagic);
+  add2g(f0, f1, x0, x1, -n0, -n1);
+  fma2g(p0, p1, f0, f1, 0.009560510516166687f, 0.009560510516166687f, 0.05591703951358795f, 0.05591703951358795f);
+  fma2g(p0, p1, p0, p1, f0, f1, 0.24024981260299683f, 0.24024981260299683f);
+  fma2g(p0, p1, p0, p1, f0, f1, 0.6931219696998596f, 0.6931219696998596f);
+  fma2g(p0, p1, p0, p1, f0, f1, 0.9999991655349731f, 0.9999991655349731f);
+  r0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
+  r1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
