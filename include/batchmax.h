@@ -55,7 +55,8 @@ typedef enum {
   BM_ERR_CAPACITY = 3, /* the call would make n exceed cap, or too many candidates        */
   BM_ERR_STATE = 4,    /* pos0 does not follow curr_id, or the sample range has unequal n */
   BM_ERR_CUDA = 5,     /* a CUDA runtime or driver call failed                            */
-  BM_ERR_TIMEOUT = 6   /* a bounded device-side wait expired (see bm_cache_status)        */
+  BM_ERR_TIMEOUT = 6,  /* a bounded device-side wait expired (see bm_cache_status)        */
+  BM_ERR_BOUNDS = 7    /* checked build only: a kernel met a row index outside its cache  */
 } bm_status_t;
 
 typedef enum { BM_F32 = 0, BM_BF16 = 1 } bm_dtype_t;
@@ -282,6 +283,21 @@ bm_status_t bm_cache_clear_status(bm_cache_t* cache, void* cuda_stream);
  * never be satisfied.  It gives up after its poll limit, writes BM_ERR_TIMEOUT to the status word and ends
  * normally; bm_cache_status then reports BM_ERR_TIMEOUT and the context stays usable.  Nothing else is touched. */
 bm_status_t bm_selftest_wait_timeout(bm_cache_t* cache, void* cuda_stream);
+
+/* ---- the checked build (the paper has no counterpart) ----
+ * libbatchmax_debug.so is the same library compiled with -DBM_DEBUG (python -m paper_2412_05693_b200.build --debug).
+ * Its kernels test every cache row index they are about to write with plain stores against the cache's capacity; a
+ * bad index is recorded as BM_ERR_BOUNDS in the device status word (bm_cache_status) and the access is skipped --
+ * nothing traps, the context stays usable.  Its arena has a 256-byte guard behind every slab (the header grows to
+ * 4096 bytes, so bm_arena_bytes / bm_max_batch differ from the ordinary build's); bm_cache_check_canaries counts the
+ * guards that no longer hold their pattern (synchronises cuda_stream).  In the ordinary build bm_debug_build returns
+ * 0 and there are no guards to damage. */
+int32_t bm_debug_build(void);
+/* Self-test of the row test: enqueue a one-thread kernel that asks it about the first row index past a cache (no
+ * memory is touched).  In the checked build bm_cache_status then reports BM_ERR_BOUNDS (clear it with
+ * bm_cache_clear_status); in the ordinary build the status word stays BM_OK. */
+bm_status_t bm_selftest_row_check(bm_cache_t* cache, void* cuda_stream);
+bm_status_t bm_cache_check_canaries(bm_cache_t* cache, int32_t* damaged /*HOST out*/, void* cuda_stream);
 
 /* ---- rows moved by compactions (measurement aid: the compaction term of the decode step's memory traffic) ----
  * While switched on for a handle, every eviction adds the number of cache rows it moves (each row = one key and one

@@ -10,6 +10,7 @@ from .binding import (  # noqa: F401
     Config,
     arena_bytes,
     cache_bytes_per_sample,
+    debug_build,
     kernel_launch_count,
     last_prefill_path,
     lib,

@@ -10,11 +10,12 @@ import os
 from dataclasses import dataclass
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libbatchmax.so")
+# BATCHMAX_LIB selects another build of the same library, e.g. the checked one (libbatchmax_debug.so)
+LIB_PATH = os.environ.get("BATCHMAX_LIB") or os.path.join(_PKG, "libbatchmax.so")
 
 BM_F32, BM_BF16 = 0, 1
 STATUS = {0: "BM_OK", 1: "BM_ERR_INVALID", 2: "BM_ERR_OOM", 3: "BM_ERR_CAPACITY", 4: "BM_ERR_STATE",
-          5: "BM_ERR_CUDA", 6: "BM_ERR_TIMEOUT"}
+          5: "BM_ERR_CUDA", 6: "BM_ERR_TIMEOUT", 7: "BM_ERR_BOUNDS"}
 
 
 class BMError(RuntimeError):
@@ -68,6 +69,9 @@ SIGNATURES = {
     "bm_cache_status": (_i32, [_vp, C.POINTER(_i32), _vp]),
     "bm_cache_clear_status": (_i32, [_vp, _vp]),
     "bm_selftest_wait_timeout": (_i32, [_vp, _vp]),
+    "bm_debug_build": (_i32, []),
+    "bm_selftest_row_check": (_i32, [_vp, _vp]),
+    "bm_cache_check_canaries": (_i32, [_vp, C.POINTER(_i32), _vp]),
     "bm_profile_enable": (_i32, [_i32]),
     "bm_profile_read": (_i32, [_i32, C.POINTER(C.c_float), C.POINTER(_i32)]),
     "bm_kernel_launch_count": (C.c_uint64, []),
@@ -160,6 +164,11 @@ def staging_bytes(cfg: Config, nsamples: int, I: int) -> int:
     c = cfg.c()
     _check(lib().bm_staging_bytes(C.byref(c), nsamples, I, C.byref(out)), "bm_staging_bytes")
     return out.value
+
+
+def debug_build() -> bool:
+    """True when the loaded library is the checked build (row-index checks in the kernels, guards behind the slabs)."""
+    return bool(lib().bm_debug_build())
 
 
 def kernel_launch_count() -> int:
@@ -381,6 +390,16 @@ class BatchMaxCache:
         sq = sq.contiguous()
         _check(lib().bm_cache_import_sum_sq(self.h, layer, sample, kv_head, _ptr(sq), _stream(stream)),
                "bm_cache_import_sum_sq")
+
+    def selftest_row_check(self, stream=None):
+        """Enqueue the row-test self-test: in the checked build status() then reports 7 (BM_ERR_BOUNDS)."""
+        _check(lib().bm_selftest_row_check(self.h, _stream(stream)), "bm_selftest_row_check")
+
+    def check_canaries(self, stream=None) -> int:
+        """Number of damaged guards behind the arena's slabs (always 0 in the ordinary build, which has none)."""
+        bad = _i32(0)
+        _check(lib().bm_cache_check_canaries(self.h, C.byref(bad), _stream(stream)), "bm_cache_check_canaries")
+        return bad.value
 
     def clear_status(self, stream=None):
         _check(lib().bm_cache_clear_status(self.h, _stream(stream)), "bm_cache_clear_status")

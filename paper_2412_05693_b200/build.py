@@ -1,6 +1,6 @@
 """Builds libbatchmax.so (the C-ABI library) in-tree with nvcc for sm_100a.
 
-    python -m paper_2412_05693_b200.build [--force] [--verbose]
+    python -m paper_2412_05693_b200.build [--force] [--verbose] [--debug]
 """
 from __future__ import annotations
 
@@ -12,6 +12,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libbatchmax.so")
+DEBUG_LIB_PATH = os.path.join(PKG_DIR, "libbatchmax_debug.so")   # the checked build: -DBM_DEBUG
 HEADER = os.path.join(os.path.dirname(PKG_DIR), "include", "batchmax.h")
 
 NVCC_FLAGS = [
@@ -24,27 +25,29 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def _stale(lib_path: str = LIB_PATH) -> bool:
+    if not os.path.exists(lib_path):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(lib_path)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + [HEADER]
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into one shared library; returns its path."""
-    if not force and not _stale():
-        return LIB_PATH
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compile every .cu under csrc/ into one shared library; returns its path.  debug: the checked build
+    (row-index checks in the kernels, guards behind the slabs), libbatchmax_debug.so."""
+    lib_path = DEBUG_LIB_PATH if debug else LIB_PATH
+    if not force and not _stale(lib_path):
+        return lib_path
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     objs = []
     procs = []
-    build_dir = os.path.join(PKG_DIR, "build")
+    build_dir = os.path.join(PKG_DIR, "build", "debug" if debug else "release")
     os.makedirs(build_dir, exist_ok=True)
     for src in sources():
         obj = os.path.join(build_dir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
-        cmd = [nvcc, *NVCC_FLAGS, "-c", src, "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, *(["-DBM_DEBUG"] if debug else []), "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
@@ -57,10 +60,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    link = [nvcc, "-shared", "-o", LIB_PATH, *objs, "-gencode", "arch=compute_100a,code=sm_100a"]
+    link = [nvcc, "-shared", "-o", lib_path, *objs, "-gencode", "arch=compute_100a,code=sm_100a"]
     subprocess.run(link, check=True)
-    return LIB_PATH
+    return lib_path
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug="--debug" in sys.argv))

@@ -53,7 +53,15 @@ bm_status_t cuda_fail(cudaError_t e) {
   return BM_ERR_CUDA;
 }
 
+#ifdef BM_DEBUG
+// checked build: room for a 256-byte canary behind each of the (up to five) slabs as well
+constexpr size_t kHeaderBytes = 4096;
+constexpr size_t kCanaryBytes = 256;
+#else
 constexpr size_t kHeaderBytes = 1024;   // status word + room to align each of the four slabs to 256 B
+constexpr size_t kCanaryBytes = 0;
+#endif
+constexpr int kCanaryByte = 0xA5;
 constexpr int kMaxCandidates = 12288;   // candidates of one eviction must fit one CTA's shared memory
 constexpr size_t kMaxSmem = 227 * 1024;
 
@@ -125,6 +133,7 @@ struct bm_cache {
   std::vector<int32_t> npad;      // [L * b] padding pairs cached (kNpadUnknown after an import / set_len)
   bool count_moves = false;      // compactions add the rows they move to the counters in the status block
   std::vector<int32_t> n, curr_id;  // [L * b] host mirror
+  std::vector<char*> canaries;      // checked build: the 256-byte guard behind each slab
   // host-fed calls run as a three-stage pipeline on streams owned by the handle -- input copies, the pass,
   // the output copy -- so that the three stages of consecutive calls overlap (PCIe is full duplex); the
   // caller's stream only waits for each call's output copy.  Up to four staging buffers can be in flight.
@@ -269,12 +278,17 @@ bm_status_t bm_cache_create(const bm_config_t* cfg, void* arena, size_t arena_by
   c->status = reinterpret_cast<int32_t*>(p);
   // header = 256 B status block + up to 3 * 256 B of slab alignment padding
   size_t off = 256;
-  c->k_slab = p + off;                                   off = align_up(off + slab, 256);
-  c->v_slab = p + off;                                   off = align_up(off + slab, 256);
-  c->sum_weights = reinterpret_cast<float*>(p + off);    off = align_up(off + rows * 4, 256);
-  c->kv_ids = reinterpret_cast<int32_t*>(p + off);       off += rows * 4;
+  auto guard = [&]() {   // checked build: a canary behind the slab that ends at `off`
+    if (kCanaryBytes > 0) { c->canaries.push_back(p + off); off += kCanaryBytes; }
+  };
+  c->k_slab = p + off;                                   off = align_up(off + slab, 256);      guard();
+  c->v_slab = p + off;                                   off = align_up(off + slab, 256);      guard();
+  c->sum_weights = reinterpret_cast<float*>(p + off);    off = align_up(off + rows * 4, 256);  guard();
+  c->kv_ids = reinterpret_cast<int32_t*>(p + off);       off = kCanaryBytes > 0 ? align_up(off + rows * 4, 256) : off + rows * 4;
+  guard();
   if (cfg->rule == BM_RULE_AVERAGE_STD) {   // a fifth slab of 4-byte entries right behind the fourth
-    c->sum_sq = reinterpret_cast<float*>(p + off);       off += rows * 4;
+    c->sum_sq = reinterpret_cast<float*>(p + off);       off = kCanaryBytes > 0 ? align_up(off + rows * 4, 256) : off + rows * 4;
+    guard();
   }
   if (off > need_arena) { delete c; return BM_ERR_OOM; }
   c->ws_lse = static_cast<float*>(workspace);
@@ -291,6 +305,11 @@ bm_status_t bm_cache_create(const bm_config_t* cfg, void* arena, size_t arena_by
     delete c;
     return BM_ERR_CUDA;
   }
+  for (char* g : c->canaries)
+    if (cudaMemsetAsync(g, kCanaryByte, kCanaryBytes, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+      delete c;
+      return BM_ERR_CUDA;
+    }
   *out = c;
   return BM_OK;
 }
@@ -743,6 +762,40 @@ bm_status_t bm_selftest_wait_timeout(bm_cache_t* c, void* cuda_stream) {
              ? BM_OK : BM_ERR_CUDA;
 }
 
+int32_t bm_debug_build(void) {
+#ifdef BM_DEBUG
+  return 1;
+#else
+  return 0;
+#endif
+}
+
+bm_status_t bm_cache_check_canaries(bm_cache_t* c, int32_t* damaged, void* cuda_stream) {
+  if (c == nullptr || damaged == nullptr) return BM_ERR_INVALID;
+  *damaged = 0;
+  bm_status_t s = set_device(c);
+  if (s != BM_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  std::vector<unsigned char> host(256);
+  for (char* g : c->canaries) {
+    if (cudaMemcpyAsync(host.data(), g, 256, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+      return BM_ERR_CUDA;
+    for (unsigned char b : host)
+      if (b != kCanaryByte) { ++*damaged; break; }
+  }
+  return BM_OK;
+}
+
+bm_status_t bm_selftest_row_check(bm_cache_t* c, void* cuda_stream) {
+  if (c == nullptr) return BM_ERR_INVALID;
+  bm_status_t s = set_device(c);
+  if (s != BM_OK) return s;
+  const CacheView view = make_view(c, 0, 0, 1, 0, false);
+  const cudaError_t e = launch_row_check_selftest(view, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? BM_OK : cuda_fail(e);
+}
+
 bm_status_t bm_profile_enable(int32_t on) {
   g_profile_on = on != 0;
   return BM_OK;
@@ -782,6 +835,7 @@ const char* bm_status_string(bm_status_t s) {
     case BM_ERR_STATE: return "call out of order for the cache state";
     case BM_ERR_CUDA: return "CUDA call failed";
     case BM_ERR_TIMEOUT: return "bounded device wait expired";
+    case BM_ERR_BOUNDS: return "a kernel of the checked build met a row index outside its cache";
     default: return "unknown status";
   }
 }

@@ -42,6 +42,20 @@ __device__ inline int sample_left_pad(const CacheView& c, int smp) {
   return c.left_pad != nullptr ? c.left_pad[smp] : 0;
 }
 
+// Checked build (-DBM_DEBUG, libbatchmax_debug.so): every cache row index a kernel is about to write with plain
+// stores is tested against the cache's capacity first; a bad index records BM_ERR_BOUNDS in the status word and the
+// access is skipped (nothing traps).  In the ordinary build the test is the constant `true`.
+constexpr int kErrBounds = 7;   // BM_ERR_BOUNDS
+#ifdef BM_DEBUG
+__device__ inline bool row_ok(const CacheView& c, long long r) {
+  if (r >= 0 && r < c.cap) return true;
+  atomicExch(c.status, kErrBounds);
+  return false;
+}
+#else
+__device__ __forceinline__ constexpr bool row_ok(const CacheView&, long long) { return true; }
+#endif
+
 // One forward pass over a block (I inputs) for the range.
 struct BlockArgs {
   const void* q;    // [nsamples][I][Hq][d]
@@ -81,6 +95,7 @@ size_t evict_smem_bytes(int n_cand, int target);
 size_t decode_smem_bytes(int d, int g, int n_rows, int target);
 bool tc_path_available();
 cudaError_t launch_wait_timeout_selftest(int* status, cudaStream_t st);
+cudaError_t launch_row_check_selftest(const CacheView& c, cudaStream_t st);
 cudaError_t launch_attn_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used);
 cudaError_t launch_score_tc(int d, const CacheView& c, const BlockArgs& a, cudaStream_t st, int* used);
 

@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
     const int pc = tid % LPR;
     const T* src = reinterpret_cast<const T*>(tid < LPR ? a.k : a.v) + ((size_t)smp * c.Hkv + kh) * D + pc * V;
     T* dst = (tid < LPR ? kslab : vslab) + (size_t)c.n_old * D + pc * V;
-    st_global_16(dst, ld_global_16(src));
+    if (row_ok(c, c.n_old)) st_global_16(dst, ld_global_16(src));
   }
   for (int j = tid; j < n1; j += kDecThreads) s.id[j] = (j < c.n_old) ? c.kv_ids[base + j] : a.pos;
   __syncthreads();
@@ -212,7 +212,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
       else if (c.rule == 0) ave = sw / ((float)G * (float)(a.pos + 1 - s.id[j]));
       else ave = (c.rule == 1 && j >= n1 - a.target / 2) ? INFINITY : sw;
       if (ave <= best_ave) { best_ave = ave; best_j = j; }   // j ascends: ties move to the higher position
-    } else {
+    } else if (row_ok(c, j)) {
       c.sum_weights[base + j] = sw;
     }
   }
@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
         const int j = j0 + u * SLOTS;
-        if (j < n1 && j > hole) st_global_16(vslab + (size_t)(j - 1) * D + lr * V, raw[u]);
+        if (j < n1 && j > hole && row_ok(c, j - 1)) st_global_16(vslab + (size_t)(j - 1) * D + lr * V, raw[u]);
       }
     }
   }
@@ -298,7 +298,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_kernel(CacheView c, Decode
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
         const int j = j0 + u * SLOTS;
-        if (j < n1 && j > hole) st_global_16(kslab + (size_t)(j - 1) * D + lr * V, raw[u]);
+        if (j < n1 && j > hole && row_ok(c, j - 1)) st_global_16(kslab + (size_t)(j - 1) * D + lr * V, raw[u]);
       }
     }
   }

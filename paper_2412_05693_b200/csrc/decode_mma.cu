@@ -157,7 +157,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
     const int pc = tid % (D / 8);
     const T* src = reinterpret_cast<const T*>(tid < D / 8 ? a.k : a.v) + ((size_t)smp * c.Hkv + kh) * D + pc * 8;
     T* dst = (tid < D / 8 ? kslab : vslab) + (size_t)c.n_old * D + pc * 8;
-    st_global_16(dst, ld_global_16(src));
+    if (row_ok(c, c.n_old)) st_global_16(dst, ld_global_16(src));
   }
   for (int j = tid; j < n1t; j += kThreads) s.id[j] = (j < c.n_old) ? c.kv_ids[base + j] : a.pos;
   // q fragments: thread (gid, tq) holds, for every pair of rounds (2R, 2R+1), the 16 elements [64R + 16tq, +16) of
@@ -383,7 +383,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
       else ave = (rule == 1 && j >= n1 - a.target / 2) ? INFINITY : sw;
       // ties: the higher position leaves (kv_ids, not rows: the rows of an unordered cache are in no order)
       if (ave < best_ave || (ave == best_ave && s.id[j] > best_id)) { best_ave = ave; best_j = j; best_id = s.id[j]; }
-    } else {
+    } else if (row_ok(c, j)) {
       c.sum_weights[base + j] = sw;
     }
   }
@@ -422,6 +422,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
       if (c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)(n1 - 1 - hole));
       // sum_weights / kv_ids in their final places: rows behind the hole move up by one
       for (int j = tid; j < n1; j += kThreads) {
+        if (!row_ok(c, j)) continue;
         if (j < hole) c.sum_weights[base + j] = s.score[j];
         else if (j > hole) { c.sum_weights[base + j - 1] = s.score[j]; c.kv_ids[base + j - 1] = s.id[j]; }
       }
@@ -471,7 +472,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
 #pragma unroll
         for (int sx = 0; sx < 4; ++sx) {
           const int j = jr + sx;
-          if (j < n1 && j > hole) st_global_16(vslab + (size_t)(j - 1) * D + 64 * r + 8 * gid, zt[r][sx]);
+          if (j < n1 && j > hole && row_ok(c, j - 1)) st_global_16(vslab + (size_t)(j - 1) * D + 64 * r + 8 * gid, zt[r][sx]);
         }
     }
   };
@@ -482,8 +483,8 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
         const int j0 = u * kRowsPerIter + warp * 16 + gid, j1 = j0 + 8;
 #pragma unroll
         for (int R = 0; R < QR / 2; ++R) {
-          if (j0 < n1 && j0 > hole) stg32(kslab + (size_t)(j0 - 1) * D + 64 * R + 16 * tq, xk[u][2 * R], xk[u][2 * R + 1]);
-          if (j1 < n1 && j1 > hole) stg32(kslab + (size_t)(j1 - 1) * D + 64 * R + 16 * tq, yk[u][2 * R], yk[u][2 * R + 1]);
+          if (j0 < n1 && j0 > hole && row_ok(c, j0 - 1)) stg32(kslab + (size_t)(j0 - 1) * D + 64 * R + 16 * tq, xk[u][2 * R], xk[u][2 * R + 1]);
+          if (j1 < n1 && j1 > hole && row_ok(c, j1 - 1)) stg32(kslab + (size_t)(j1 - 1) * D + 64 * R + 16 * tq, yk[u][2 * R], yk[u][2 * R + 1]);
         }
       }
     }
@@ -510,11 +511,11 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
       const int pieces = (min(r8, n1) - 1 - hole) * (D / 8);
       if (tid < pieces) {
         const int j = hole + 1 + tid / (D / 8), pc = tid % (D / 8);
-        st_global_16(vslab + (size_t)(j - 1) * D + pc * 8, *v_piece(j, pc));
+        if (row_ok(c, j - 1)) st_global_16(vslab + (size_t)(j - 1) * D + pc * 8, *v_piece(j, pc));
       }
       for (int x = tid; x < (n1 - r_tail) * (D / 8); x += kThreads) {
         const int j = r_tail + x / (D / 8), pc = x % (D / 8);
-        st_global_16(vslab + (size_t)(j - 1) * D + pc * 8, *v_piece(j, pc));
+        if (row_ok(c, j - 1)) st_global_16(vslab + (size_t)(j - 1) * D + pc * 8, *v_piece(j, pc));
       }
       if (tid == 0) {
         for (int r0 = r8; r0 < min(n1, r_tail); r0 += 128) {
@@ -568,7 +569,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
     if (hole < c.n_old && tid < 2 * (D / 8)) {
       const int pc = tid % (D / 8);
       T* dst = (tid < D / 8 ? kslab : vslab) + (size_t)hole * D + pc * 8;
-      st_global_16(dst, ld_global_16((tid < D / 8 ? k_new : v_new) + pc * 8));
+      if (row_ok(c, hole)) st_global_16(dst, ld_global_16((tid < D / 8 ? k_new : v_new) + pc * 8));
     }
   } else if (KD == 1 && evict_one) {
     constexpr int PR = D / 8;                 // 16-byte pieces per row
@@ -585,7 +586,7 @@ __global__ void __launch_bounds__(NT, KD > 1 ? 1 : 512 / NT) decode_mma_kernel(C
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const int j = r0 + slot + u * (kThreads / PR);
-        if (j < n1 && j > hole) st_global_16(kslab + (size_t)(j - 1) * D + pc * 8, raw[u]);
+        if (j < n1 && j > hole && row_ok(c, j - 1)) st_global_16(kslab + (size_t)(j - 1) * D + pc * 8, raw[u]);
       }
     }
   }

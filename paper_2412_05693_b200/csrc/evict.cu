@@ -32,6 +32,15 @@ cudaError_t launch_t(const CacheView& c, const EvictArgs& e, cudaStream_t st) {
 
 }  // namespace
 
+// Self-test of the checked build's row test: asks it about the first row index past the cache (nothing is accessed).
+__global__ void row_check_selftest(CacheView c) { (void)row_ok(c, c.cap); }
+
+cudaError_t launch_row_check_selftest(const CacheView& c, cudaStream_t st) {
+  row_check_selftest<<<1, 1, 0, st>>>(c);
+  count_launch();
+  return cudaGetLastError();
+}
+
 size_t evict_smem_bytes(int n_cand, int target) { return evict_smem_layout(nullptr, n_cand, target, nullptr); }
 
 cudaError_t launch_evict(int dtype, int d, const CacheView& c, const EvictArgs& e, cudaStream_t st) {

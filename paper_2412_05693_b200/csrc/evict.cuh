@@ -172,6 +172,7 @@ __device__ inline void evict_body_impl(const CacheView& c, int unit, int smp, in
     if (c.moved != nullptr && tid == 0) atomicAdd(&c.moved[unit & 15], (unsigned long long)nf);
     for (int k = tid; k < nf; k += NT) {
       const int j = s.src[k], r = s.dst[k];
+      if (!row_ok(c, r)) continue;
       c.sum_weights[base + r] = s.score[j];
       c.kv_ids[base + r] = s.id[j];
     }
@@ -201,6 +202,7 @@ __device__ inline void evict_body_impl(const CacheView& c, int unit, int smp, in
         const int x = x0 + t * NT + tid;
         if (x < nf * PRF) {
           const int r = s.dst[x / PRF], pc = x % PRF;
+          if (!row_ok(c, r)) continue;
           st_global_16(kslab + (size_t)r * D + pc * (16 / sizeof(T)), kb[t]);
           st_global_16(vslab + (size_t)r * D + pc * (16 / sizeof(T)), vb[t]);
         }
@@ -319,6 +321,7 @@ __device__ inline void evict_body_impl(const CacheView& c, int unit, int smp, in
 
   for (int r = first_moved + tid; r < target; r += NT) {
     const int j = s.src[r];
+    if (!row_ok(c, r) || j < 0 || j >= n_c) continue;
     c.sum_weights[base + r] = s.score[j];
     c.kv_ids[base + r] = s.id[j];
   }
@@ -328,7 +331,8 @@ __device__ inline void evict_body_impl(const CacheView& c, int unit, int smp, in
     for (int j = tid; j < n_c; j += NT)
       s.bits[j] = __float_as_uint(j < n_old ? c.sum_sq[base + j] : e.new_sq[(size_t)unit * e.I + (j - n_old)]);
     __syncthreads();
-    for (int r = first_moved + tid; r < target; r += NT) c.sum_sq[base + r] = __uint_as_float(s.bits[s.src[r]]);
+    for (int r = first_moved + tid; r < target; r += NT)
+      if (row_ok(c, r)) c.sum_sq[base + r] = __uint_as_float(s.bits[s.src[r]]);
   }
 
   // ---- rows: ascending chunks, every source row index >= its destination, loads of a chunk complete
@@ -364,6 +368,7 @@ __device__ inline void evict_body_impl(const CacheView& c, int unit, int smp, in
     for (int t = 0; t < U; ++t) {
       if (mv[t]) {
         const int pidx = t * NT + tid, r = r0 + pidx / PR, pc = pidx % PR;
+        if (!row_ok(c, r)) continue;
         st_global_16(kslab + (size_t)r * D + pc * (16 / sizeof(T)), kb[t]);
         st_global_16(vslab + (size_t)r * D + pc * (16 / sizeof(T)), vb[t]);
       }

@@ -215,6 +215,9 @@ def run_lockstep(wl: Workload, units, device: int = 0, layer: int = 0, calls=Non
             if want_rows:
                 assert np.array_equal(_np(kr), unit.k), f"{where}: cached K rows are not the oracle's rows"
                 assert np.array_equal(_np(vr), unit.v), f"{where}: cached V rows are not the oracle's rows"
+    from paper_2412_05693_b200 import debug_build
+    if debug_build():                               # the checked build: no guard behind a slab was written over
+        assert cache.check_canaries() == 0, "a guard behind one of the arena's slabs was damaged"
     if own_cache:
         cache.close()
     return stats

@@ -34,6 +34,22 @@ def test_library_exports_every_declared_symbol():
     assert set(names) == set(binding.SIGNATURES), "binding and header disagree on the entry points"
 
 
+def test_checked_build_exports_the_same_symbols_and_charges_its_guards():
+    # libbatchmax_debug.so: same entry points; its arena header holds a 256-byte guard behind every slab
+    h = C.CDLL(build(debug=True))
+    for n in declared_symbols():
+        assert hasattr(h, n), f"{n} missing from the checked build"
+    h.bm_debug_build.restype = C.c_int32
+    assert h.bm_debug_build() == 1 and bm.lib().bm_debug_build() == 0
+    cfg = llama_cfg().c()
+    need = C.c_size_t(0)
+    h.bm_arena_bytes.argtypes = [C.POINTER(binding.bm_config_t), C.POINTER(C.c_size_t)]
+    assert h.bm_arena_bytes(C.byref(cfg), C.byref(need)) == 0
+    assert need.value == 4096 + 16 * 8 * 1025 * 520
+    # the memory model also charges the rule that keeps a second accumulator per row
+    assert bm.cache_bytes_per_sample(llama_cfg(rule="average_std")) == 8 * 1025 * (2 * 128 * 2 + 12)
+
+
 def llama_cfg(**kw):
     base = dict(batch=16, n_q_heads=32, n_kv_heads=8, head_dim=128, kv_max=1024, block_max=512, growth=1)
     base.update(kw)
