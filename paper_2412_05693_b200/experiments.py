@@ -189,7 +189,10 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
     moved_pre = None
     ms_pre = ms_dec = 0.0
     layers = range(wl.L) if layers is None else layers
-    out_blk = torch.empty(micro, cfg.block_max, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
+    out_flat = torch.empty(micro * cfg.block_max * wl.Hq * wl.d, dtype=wl.torch_dtype, device=dev)
+
+    def out_blk(ns, I):     # a contiguous (ns, I, Hq, d) view: the library writes the output with q's layout
+        return out_flat[:ns * I * wl.Hq * wl.d].view(ns, I, wl.Hq, wl.d)
     micro_dec = max(micro, min(batch, DECODE_MICRO))
     out_dec = torch.empty(micro_dec, wl.Hq, wl.d, dtype=wl.torch_dtype, device=dev)
     calls = arm_calls(wl, arm, kv_bar, p)
@@ -214,7 +217,7 @@ def run_arm(wl: Workload, batch: int, arm: str, micro: int, arena=None, layers=N
                 for s0 in range(0, batch, micro):
                     ns = min(micro, batch - s0)
                     q, k, v = inp.block(layer, pos0, I, s0, ns)
-                    timer(lambda: cache.prefill_block(q, k, v, pos0, out=out_blk[:ns, :I], evict_to=arg, layer=layer,
+                    timer(lambda: cache.prefill_block(q, k, v, pos0, out=out_blk(ns, I), evict_to=arg, layer=layer,
                                                       sample0=s0))
                 pairs += I * n + I * (I + 1) // 2
                 n = n + I if arg < 0 else min(n + I, arg)
