@@ -746,9 +746,10 @@ def test_sample_ranges_on_concurrent_streams_match_whole_batch_calls(compaction)
             assert all(torch.equal(a, b) for a, b in zip(got, want)), f"{R} ranges: cache state differs"
 
 
-def test_export_import_roundtrip_resumes_identically():
+@pytest.mark.parametrize("rule", ["average", "average_std"])
+def test_export_import_roundtrip_resumes_identically(rule):
     wl = tiny("ckpt", dtype="bf16", d=128, Hq=8, Hkv=2, s=192, B=64, K=48, steps=0)
-    cfg = make_config(wl)
+    cfg = make_config(wl, rule=rule)
     inp = Inputs(wl, "cuda")
     a = bm.BatchMaxCache(cfg)
     for kind, pos0, I, ev in schedule(wl)[:2]:
@@ -759,6 +760,8 @@ def test_export_import_roundtrip_resumes_identically():
         b.set_len(n, cur, sample=s)
         for h in range(wl.Hkv):
             b.import_(*a.export(0, s, h, rows=True), sample=s, kv_head=h)
+            if rule == "average_std":       # the rule's second accumulator travels on its own pair of calls
+                b.import_sum_sq(a.export_sum_sq(0, s, h), sample=s, kv_head=h)
     kind, pos0, I, ev = schedule(wl)[2]
     q, k, v = inp.block(0, pos0, I)
     oa, ob = a.prefill_block(q, k, v, pos0, evict_to=ev), b.prefill_block(q, k, v, pos0, evict_to=ev)
@@ -767,6 +770,8 @@ def test_export_import_roundtrip_resumes_identically():
         for h in range(wl.Hkv):
             for x, y in zip(a.export(0, s, h, rows=True), b.export(0, s, h, rows=True)):
                 assert torch.equal(x, y)
+            if rule == "average_std":
+                assert torch.equal(a.export_sum_sq(0, s, h), b.export_sum_sq(0, s, h))
 
 
 def test_batch_sized_by_the_allocator_fits_its_arena():
