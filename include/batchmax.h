@@ -87,8 +87,8 @@ typedef enum { BM_F32 = 0, BM_BF16 = 1 } bm_dtype_t;
 typedef enum { BM_RULE_AVERAGE = 0, BM_RULE_SUM_RECENT = 1, BM_RULE_CURRENT_QUERY = 2, BM_RULE_WINDOW_POOLED = 3,
                BM_RULE_AVERAGE_STD = 4 } bm_rule_t;
 
-/* What "remove pairs" does to the rows of a cache.  Attention, the scores and the kept sets do not depend on the
- * order of a cache's rows; only the work of removing does.
+/* What the removal step of Algorithm 1 does to the rows of a cache.  Attention, the scores and the kept sets do not
+ * depend on the order of a cache's rows; only the work of removing does.
  *   BM_COMPACT_STABLE: rows stay in ascending kv_ids order; the rows behind a pair that leaves move up.
  *   BM_COMPACT_FILL:   rows are an unordered set: a pair that stays never moves, the pairs that arrive (the block's
  *                      kept pairs, the decode step's pair) take the rows that were freed.  Kept sets, sum_weights and

@@ -1,4 +1,4 @@
-// One decoding step (Algorithm 1 "generate token", Sec. 3.2 with I = 1) for every (sample, kv-head)
+// One decoding step (the token-generation step of Algorithm 1; Sec. 3.2 with I = 1) for every (sample, kv-head)
 // cache of a range, in one bandwidth-bound pass per cache (one CTA):
 //   append the step's pair -> logits (K streamed once for the g heads, 128-bit loads) -> softmax ->
 //   sum_weights update -> choice of the pair to evict -> P.V (V streamed once) with the one-row

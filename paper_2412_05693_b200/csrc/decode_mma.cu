@@ -1,4 +1,4 @@
-// bf16 decoding step (Algorithm 1 "generate token", Sec. 3.2 with I = 1), one CTA per (sample, kv-head) cache.
+// bf16 decoding step (the token-generation step of Algorithm 1; Sec. 3.2 with I = 1), one CTA per (sample, kv-head) cache.
 // Same steps as the fp32 kernel in decode.cu, but the two contractions run on warp-level tensor-core MMAs
 // (m16n8k16, bf16 in, fp32 accumulate) fed straight from 128-bit global loads, so that the kernel issues few
 // enough instructions to be limited by HBM bandwidth:
