@@ -38,8 +38,14 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* b) {
 // kernel's instructions).
 __device__ __forceinline__ void mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag, int* status,
                                           int limit = kWaitLimit) {
-  if (*abort_flag) return;
   const uint32_t addr = smem_u32(b);
+  {   // the phase is often complete already: one plain test before anything else
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.b32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(addr), "r"(parity) : "memory");
+    if (ok) return;
+  }
+  if (*abort_flag) return;
   for (int it = 0; it < limit; ++it) {
     uint32_t ok;
     asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\nselp.b32 %0, 1, 0, p;\n}\n"
